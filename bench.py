@@ -34,9 +34,9 @@ from paper_2602_17681_b200 import synth  # noqa: E402
 
 FMT_RATIO_TO_BF16 = {"mxfp4": 4.0, "mxfp8": 2.0, "mxint8": 1.0, "mxint4": 2.0}   # nominal dense tensor-rate ratios on B200
 METRIC = "fused transform+MX linear throughput"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture summarised in
-# profiles/mx_gemm_pair_tc_kernel_cfg2_gate_up.md (same command, same kernel); other workloads were not captured.
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_gate_up": 220.4e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from an ncu capture of this command
+# with the kernel as it is now; None = not captured (or the kernel has changed since the counters were taken).
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_gate_up": None}
 
 
 def load_peaks():
@@ -46,6 +46,18 @@ def load_peaks():
             p = json.load(f)
         return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"], source="measured")
     return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def pick_regime(clocks, region_ms):
+    """Which measured peak a timing belongs with.  "sustained": the power cap was active, or a region long enough to
+    be sampled ran with the SM clock well below its maximum; "burst" otherwise (a short region at full clock).  Without
+    usable clock samples the burst figure, the larger one, is taken, so that a fraction is never flattered."""
+    sm, smax = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    if "sw_power_cap" in (clocks.get("reasons") or []):
+        return "sustained"
+    if sm is None or not smax or region_ms < 100.0:
+        return "burst"
+    return "sustained" if sm < 0.9 * smax else "burst"
 
 
 def layer_flops(M, K, N, transform="full"):
@@ -268,6 +280,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     status = B.device_status(ws)
     if status != B.OK:
         raise RuntimeError(f"device status after timed region: {B.status_string(status)}")
+    clocks = sampler.stop()
     ms_step = ms_total / args.steps
     f1, f3 = layer_flops(M, K, N, args.transform)
     value = world * (f1 + f3) / (ms_step * 1e-3) / 1e12
@@ -276,52 +289,88 @@ def run_ours(args, cfg, rank, world, local_rank):
     a_codes, a_scales = B.alloc_mx(M, K, fmt, B.SF_TCGEN05, dev)
     k_iters = max(10, min(args.steps, 200))
     e = [torch.cuda.Event(enable_timing=True) for _ in range(3 * k_iters)]
-    for i in range(k_iters):
-        s = sets[i % n_sets]
-        e[3 * i].record()
-        B.quantize_mx(s["X"], s["A"], s["b"], fmt, B.SF_TCGEN05, ws=ws, out=(a_codes, a_scales), flags=flags)
-        e[3 * i + 1].record()
-        B.mx_gemm(a_codes, a_scales, s["Wq"], s["Wsc"], s["c"], M, K, N, fmt, out=s["out"], ws=ws)
-        e[3 * i + 2].record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
+    sampler_k = ClockSampler(local_rank)
+    sampler_k.start()
+    for rep in range(2 if k_iters < 100 else 1):         # a short run is repeated so that the clock sampler sees it
+        for i in range(k_iters):
+            s = sets[i % n_sets]
+            e[3 * i].record()
+            B.quantize_mx(s["X"], s["A"], s["b"], fmt, B.SF_TCGEN05, ws=ws, out=(a_codes, a_scales), flags=flags)
+            e[3 * i + 1].record()
+            B.mx_gemm(a_codes, a_scales, s["Wq"], s["Wsc"], s["c"], M, K, N, fmt, out=s["out"], ws=ws)
+            e[3 * i + 2].record()
+        torch.cuda.synchronize()
+    clocks_k = sampler_k.stop()
     t_k1 = float(np.mean([e[3 * i].elapsed_time(e[3 * i + 1]) for i in range(k_iters)]))
     t_k2 = float(np.mean([e[3 * i + 1].elapsed_time(e[3 * i + 2]) for i in range(k_iters)]))
 
-    p_bf16 = peaks["bf16_sustained"]
-    p_mx = p_bf16 * FMT_RATIO_TO_BF16[cfg.fmt]
+    # ---- the tensor pipes' own rate: back-to-back MMAs on operands resident in shared memory, all SMs
+    pipe = None
+    if not args.no_pipe_probe:
+        pipe = {kind: B.tensor_pipe_probe(kind, ws=ws) for kind in ("bf16", "mxf8", "mxf4")}
+
+    # Each time is compared with the measured peak of the regime it was taken in: the burst figure when the SM clock sat
+    # near its maximum, the sustained one when the power cap held it down; both fractions are printed.
+    ratio = FMT_RATIO_TO_BF16[cfg.fmt]
+    bf16 = {"burst": peaks["bf16_burst"], "sustained": peaks["bf16_sustained"]}
+    regime = pick_regime(clocks, ms_total)
+    regime_k = pick_regime(clocks_k, (t_k1 + t_k2) * k_iters * (2 if k_iters < 100 else 1))
     byts = layer_bytes(M, K, N, cfg.fmt, args.transform)
-    if args.transform == "full":
-        t1_s = f1 / (p_bf16 * 1e12)
-    else:   # the block-wise transform is bound by reading X and writing codes and scales
-        t1_s = (2.0 * M * K + M * K * ((0.5 if cfg.fmt == "mxfp4" else 1.0) + 1 / 32.0)) / (peaks["hbm_gbs"] * 1e9)
-    r2_ms = max(t1_s + f3 / (p_mx * 1e12), byts / (peaks["hbm_gbs"] * 1e9)) * 1e3
-    r1_ms = max((f1 + f3) / (p_mx * 1e12), byts / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    hbm_s = byts / (peaks["hbm_gbs"] * 1e9)
+
+    def layer_rooflines(p_bf16):
+        if args.transform == "full":
+            t1_s = f1 / (p_bf16 * 1e12)
+        else:   # the block-wise transform is bound by reading X and writing codes and scales
+            t1_s = (2.0 * M * K + M * K * ((0.5 if cfg.fmt == "mxfp4" else 1.0) + 1 / 32.0)) / (peaks["hbm_gbs"] * 1e9)
+        r2 = max(t1_s + f3 / (p_bf16 * ratio * 1e12), hbm_s) * 1e3
+        r1 = max((f1 + f3) / (p_bf16 * ratio * 1e12), hbm_s) * 1e3
+        return r2, r1
+    r2_ms, r1_ms = layer_rooflines(bf16[regime])
+    k1_tflops = f1 / (t_k1 * 1e-3) / 1e12
     k2_tflops = f3 / (t_k2 * 1e-3) / 1e12
+    p_mx = bf16[regime_k] * ratio
     if M > 128:
         kernel = "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)" if cfg.fmt == "mxint8" else "mx_gemm_pair_tc_kernel (block-scaled GEMM)"
     elif cfg.fmt == "mxint8":
         kernel = "mxint8_gemm_decode_tc_kernel (int8 -> bf16 in shared memory)" if M <= 16 else "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)"
     else:
         kernel = "mx_gemm_decode_tc_kernel (block-scaled GEMM, operands swapped)" if M <= 64 else "mx_gemm_tc_kernel (block-scaled GEMM)"
+    mhz_k = clocks_k.get("sm_mhz")
     roofline = {
         "bound": "tensor", "kernel": kernel,
         "achieved": k2_tflops, "peak": p_mx, "unit": "TFLOP/s", "frac": k2_tflops / p_mx,
         "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
-        "peak_source": f"{FMT_RATIO_TO_BF16[cfg.fmt]:g} x bf16 sustained {p_bf16:g} TFLOP/s of {peaks['source']} (nominal ratio)",
-        "layer": {"r2_ms": r2_ms, "r2_frac": r2_ms / ms_step, "r1_ms": r1_ms, "r1_frac": r1_ms / ms_step,
-                  "hbm_ms": byts / (peaks["hbm_gbs"] * 1e9) * 1e3, "algorithmic_bytes": byts},
-        "kernels": {"transform_quant_ms": t_k1, "transform_quant_tflops": f1 / (t_k1 * 1e-3) / 1e12,
-                    "transform_quant_frac_of_bf16_peak": f1 / (t_k1 * 1e-3) / 1e12 / p_bf16,
+        "regime": regime_k,
+        "peak_source": f"{ratio:g} x bf16 {regime_k} {bf16[regime_k]:g} TFLOP/s of {peaks['source']} (nominal ratio); "
+                       f"regime chosen from the SM clock sampled while the kernels were timed",
+        "frac_of_burst_peak": k2_tflops / (bf16["burst"] * ratio), "frac_of_sustained_peak": k2_tflops / (bf16["sustained"] * ratio),
+        "flops_per_launch": f3, "ms_per_launch": t_k2,
+        "cycles_per_launch": t_k2 * 1e-3 * mhz_k * 1e6 if mhz_k else None,
+        "clocks_kernels": clocks_k,
+        "layer": {"regime": regime, "r2_ms": r2_ms, "r2_frac": r2_ms / ms_step, "r1_ms": r1_ms, "r1_frac": r1_ms / ms_step,
+                  "r2_frac_of_burst_peaks": layer_rooflines(bf16["burst"])[0] / ms_step,
+                  "r2_frac_of_sustained_peaks": layer_rooflines(bf16["sustained"])[0] / ms_step,
+                  "hbm_ms": hbm_s * 1e3, "algorithmic_bytes": byts},
+        "kernels": {"transform_quant_ms": t_k1, "transform_quant_tflops": k1_tflops,
+                    "transform_quant_frac_of_bf16_peak": k1_tflops / bf16[regime_k],
+                    "transform_quant_frac_of_bf16_burst": k1_tflops / bf16["burst"],
                     "mx_gemm_ms": t_k2, "mx_gemm_tflops": k2_tflops},
     }
+    if pipe is not None:
+        own = {"mxfp4": "mxf4", "mxfp8": "mxf8", "mxint4": "mxf8", "mxint8": "bf16"}[cfg.fmt]
+        roofline["pipe_probe"] = {"tflops": pipe, "frac_of_probe": k2_tflops / pipe[own], "kind": own,
+                                  "note": "back-to-back tcgen05.mma 128 x 256 on shared-memory operands, every SM, about 2 ms "
+                                          "per kind, at the clock the probe itself ran at"}
     if M <= 64:
         # small batches: the dominant kernel streams the weights once; algorithmic bytes = codes + scales of both operands + result
         code = 0.5 if cfg.fmt == "mxfp4" else 1.0
         k2_bytes = (N + M) * K * (code + 1 / 32.0) + 4.0 * M * N
         gbs = k2_bytes / (t_k2 * 1e-3) / 1e9
         roofline.update({"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                         "peak_source": f"copy bandwidth of {peaks['source']}"})
+                         "peak_source": f"copy bandwidth of {peaks['source']}", "bytes_per_launch": k2_bytes})
+        for key in ("frac_of_burst_peak", "frac_of_sustained_peak", "flops_per_launch", "pipe_probe"):
+            roofline.pop(key, None)
 
     # ---- end to end through the public call with HOST buffers (pinned), copies inside the timed region
     e2e = None
@@ -448,7 +497,8 @@ def run_fold(args, cfg, local_rank):
     ms = ev0.elapsed_time(ev1) / steps
     if B.device_status(ws) != B.OK:
         raise RuntimeError("device status after timed region")
-    peak = peaks["bf16_sustained"]
+    regime = pick_regime(clocks, ms * steps)
+    peak = peaks["bf16_" + regime]
     print(json.dumps({
         "metric": "transformation MSE diagnostic time" if args.op == "mse" else "offline fold + weight quantisation time", "value": ms, "unit": "ms", "n_gpus": 1, "steps": steps,
         "warmup": warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
@@ -458,8 +508,9 @@ def run_fold(args, cfg, local_rank):
         "clocks": clocks, "gpu_launches": int(B.launch_count() - n0),
         "roofline": {"bound": "tensor", "achieved": issued / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                      "frac": issued / (ms * 1e-3) / 1e12 / peak, "traffic": None,
-                     "note": "issued bf16 flops (three-term splits) of all kernels of the call over bf16 %s sustained peak; "
-                             "algorithmic rate %.1f TFLOP/s" % (peaks["source"], flops / (ms * 1e-3) / 1e12)},
+                     "regime": regime,
+                     "note": "issued bf16 flops (three-term splits) of all kernels of the call over the bf16 %s %s peak; "
+                             "algorithmic rate %.1f TFLOP/s" % (peaks["source"], regime, flops / (ms * 1e-3) / 1e12)},
     }), flush=True)
 
 
@@ -510,6 +561,72 @@ def run_quantize(args, cfg, local_rank):
     }), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------------
+# Tensor-pipe issue-rate probe (--op mma_peak): what the pipes deliver when nothing but MMAs runs
+# ----------------------------------------------------------------------------------------------------
+def run_mma_peak(args, local_rank):
+    from paper_2602_17681_b200 import binding as B
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+    ws = B.new_workspace(B.OP_QUANTIZE_MX, 0, 64, 0, B.MXFP4, dev)
+    nominal = {"bf16": 1.0, "mxf8": 2.0, "mxf4": 4.0, "nvf4": 4.0}
+    for kind in nominal:                                   # warm-up
+        B.tensor_pipe_probe(kind, ws=ws)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    n0 = B.launch_count()
+    reps = max(3, min(args.steps, 50))
+    out = {k: max(B.tensor_pipe_probe(k, ws=ws) for _ in range(reps)) for k in nominal}
+    long_run = {k: B.tensor_pipe_probe(k, ws=ws, mma_per_cta=1 << 22) for k in ("bf16", "mxf4")}   # about 0.3 s each
+    clocks = sampler.stop()
+    print(json.dumps({
+        "metric": "tensor pipe issue rate", "value": out["mxf4"], "unit": "TFLOP/s", "n_gpus": 1, "steps": reps, "warmup": 1,
+        "higher_is_better": True, "vs_baseline": None, "dtype": "mxf4 / mxf8f6f4 / bf16 / mxf4nvf4", "data": "synthetic",
+        "config": {"workload": "back-to-back tcgen05.mma 128 x 256 x (16 | 32 | 64), operands resident in shared memory, "
+                               "one CTA per SM, best of %d launches of about 2 ms" % reps, "op": args.op},
+        "clocks": clocks, "gpu_launches": int(B.launch_count() - n0),
+        "tflops": out, "tflops_long_run": long_run,
+        "ratio_to_bf16_probe": {k: out[k] / out["bf16"] for k in out},
+        "measured_cublas_bf16": {"burst": peaks["bf16_burst"], "sustained": peaks["bf16_sustained"], "source": peaks["source"]},
+        "nominal_ratio_to_bf16": nominal,
+    }), flush=True)
+
+
+def spawn_ranks(args):
+    """`bench.py --gpus N` without a launcher: start N ranks of this same command under torch.distributed.run (one per
+    GPU, rendezvous on 127.0.0.1) and return its exit code.  Refuses when fewer than N GPUs are visible."""
+    if not args.plumbing_only and args.impl == "ours":
+        have = torch.cuda.device_count()
+        if have < args.gpus:
+            sys.stderr.write(f"bench.py: --gpus {args.gpus} asked for but {have} GPU(s) visible; not running on fewer\n")
+            return 2
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_plumbing(args, rank, world):
+    """The multi-rank plumbing without a GPU: rendezvous on gloo, barrier, row shards, max-over-ranks of a per-rank time."""
+    import torch.distributed as dist
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+        dist.barrier()
+    lo, hi = shard_rows(synth.CONFIGS[args.workload].M * world, rank, world)
+    ms = reduce_max_time(1.0 + rank, world)
+    rows = torch.tensor([hi - lo], dtype=torch.int64)
+    if world > 1:
+        dist.all_reduce(rows)
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"plumbing_only": True, "n_gpus": world, "ms_slowest_rank": ms, "rows_total": int(rows.item())}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -518,22 +635,41 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_gate_up", choices=sorted(synth.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-pipe-probe", action="store_true", help="skip the tensor-pipe issue-rate probe")
     ap.add_argument("--graph", action="store_true", help="record each step in a CUDA graph and time the replays (small batches are launch-bound)")
     ap.add_argument("--transform", default="full", choices=["full", "blockdiag"],
                     help="full K x K learned-style matrix (the configuration the metric is quoted on) or the paper's online "
                          "block transform T3 (32 x 32 Hadamard blocks)")
     ap.add_argument("--weights", default="bf16", choices=["bf16", "f32"], help="--op fold: dtype of the unfolded weights")
-    ap.add_argument("--op", default="layer", choices=["layer", "fold", "fold_two_sided", "mse", "quantize"],
+    ap.add_argument("--op", default="layer", choices=["layer", "fold", "fold_two_sided", "mse", "quantize", "mma_peak"],
                     help="layer: the online path (the metric); fold / fold_two_sided: time the offline weight preparation; "
-                         "mse: time the transformation-MSE diagnostic; quantize: the standalone quantiser (no transform)")
+                         "mse: the transformation-MSE diagnostic (time and values); quantize: the standalone quantiser (no "
+                         "transform); mma_peak: issue-rate probe of the tensor pipes")
+    ap.add_argument("--plumbing-only", action="store_true",
+                    help="no GPU work: run only the launch, rendezvous (gloo), barrier and max-over-ranks plumbing of --gpus N")
+    ap.add_argument("--block", type=int, default=32, help="--op mse: block size B of the quantiser (8, 16, 32, 64 or 128)")
+    ap.add_argument("--mse-transform", default="full", choices=["identity", "full", "hadamard"],
+                    help="--op mse: no transform, the full learned-style matrix, or 32 x 32 Hadamard blocks")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = synth.CONFIGS[args.workload]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)\n")
+        sys.exit(2)
+    if args.plumbing_only:
+        run_plumbing(args, rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
+        return
+    if args.op == "mma_peak":
+        if rank == 0:
+            run_mma_peak(args, local_rank)
         return
     if args.op != "layer":
         if rank == 0:
@@ -542,6 +678,9 @@ def main():
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if torch.cuda.device_count() < world:
+            sys.stderr.write(f"bench.py: {world} ranks but only {torch.cuda.device_count()} GPU(s) visible\n")
+            sys.exit(2)
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     try:

@@ -72,8 +72,11 @@ typedef enum {
     LATMIX_SF_LINEAR = 0,  /* [rows][K/32], byte (r, kb) at r * (K/32) + kb */
     LATMIX_SF_TCGEN05 = 1  /* tiles of 128 rows x 4 blocks = 512 bytes, ordered row-tile-major then k-tile;
                               inside a tile byte (r, kb) sits at (r % 32) * 16 + ((r % 128) / 32) * 4 + kb % 4.
-                              Rows are padded to a multiple of 128 and blocks to a multiple of 8; padding bytes
-                              are written as 0.  This is the layout the block-scaled tensor-core GEMM reads. */
+                              Rows are padded to a multiple of 128 and blocks to a multiple of 8.  When K/32 is not
+                              a multiple of 8 the whole buffer is zeroed before the scales are written; otherwise
+                              the bytes of padding rows keep what the buffer held (they scale rows or columns
+                              outside the result, which are never stored).  This is the layout the block-scaled
+                              tensor-core GEMM reads. */
 } latmix_sf_layout_t;
 
 /* Which call a workspace is sized for. */
@@ -87,10 +90,14 @@ enum {
     LATMIX_FLAG_NONE = 0,
     LATMIX_FLAG_CHECK_FINITE = 1,  /* quantiser records LATMIX_ERR_NONFINITE in the status word on NaN/Inf input */
     LATMIX_FLAG_FORCE_SIMT = 2,    /* use the plain CUDA-core kernels even where a tensor-core kernel applies */
-    LATMIX_FLAG_BLOCK_DIAG = 4     /* latmix_quantize_mx / latmix_linear: A is block-diagonal with 32 x 32 blocks that
+    LATMIX_FLAG_BLOCK_DIAG = 4,    /* latmix_quantize_mx / latmix_linear: A is block-diagonal with 32 x 32 blocks that
                                       coincide with the MX blocks (the paper's online transform T_3, a block Hadamard
                                       there); A then points to K/32 blocks [K/32][32][32], block i acting on elements
                                       32 i .. 32 i + 31:  Y[:, block i] = X[:, block i] A_i + b[block i] */
+    LATMIX_FLAG_TEST_DROP_LOAD = 1 << 16  /* for tests of the failure path only: the single-CTA block-scaled product (kernel
+                                      selection 1-3 below) leaves out the loads of the second 128-byte K slab of output tile
+                                      0, so that the waits for them expire and the call ends with LATMIX_ERR_TIMEOUT in the
+                                      status word; tile 0's part of `out` is then not written */
 };
 /* Bits 8-11 of `flags` select a kernel where several apply (for tests and measurements; results agree bit for bit in the
  * block-scaled product, up to near-ties in the transform): 0 = the library's choice by shape, 1-3 = single-CTA tensor-core
@@ -172,7 +179,8 @@ latmix_status_t latmix_fold_weights_two_sided(const float* A_in_inv, const float
  * With bf16 inputs the product runs on the tensor cores (bf16 x bf16 -> fp32); with fp32 inputs it is an
  * fp32 FMA product.  The accumulated fp32 value is quantised directly (never rounded to bf16 first).
  * With LATMIX_FLAG_BLOCK_DIAG, A holds K/32 blocks of 32 x 32 (same dtype as X) and the transform costs 64 flops per
- * element instead of 2 K: an fp32 FMA product fused with the quantiser, bound by reading X.
+ * element instead of 2 K: with bf16 inputs and K a multiple of 128 a warp-level tensor-core product (mma.sync, the blocks
+ * held in registers), otherwise an fp32 FMA product; either way fused with the quantiser and bound by reading X.
  */
 latmix_status_t latmix_quantize_mx(const void* X, latmix_dtype_t x_dtype, const void* A, const float* b,
                                    int64_t M, int64_t K, latmix_format_t fmt, latmix_sf_layout_t sf,
@@ -250,8 +258,29 @@ latmix_status_t latmix_linear_static(const void* X, latmix_dtype_t x_dtype, cons
                                      int64_t K, int64_t N, latmix_format_t fmt, float* out, int64_t ldo,
                                      uint32_t flags, latmix_status_t* device_status, void* cuda_stream);
 
-/* Zero the status word of a workspace (enqueued on the stream).  Call once after allocating it. */
+/*
+ * Measurement aid (the paper has no counterpart; its Sec. 5.3 reports throughput only end to end): the rate at which the
+ * tensor pipes retire MMAs when nothing else limits them.  One CTA per SM issues `mma_per_cta` (rounded down to a
+ * multiple of 4; 4 .. 2^22) tcgen05.mma of shape 128 x 256 x k back to back on operands that sit in shared memory; the
+ * results are discarded.  kind: 0 = kind::f16 with bf16 operands (k = 16), 1 = kind::mxf8f6f4 with E4M3 elements and E8M0
+ * block scales (k = 32), 2 = kind::mxf4 with E2M1 elements and E8M0 block scales (k = 64), 3 = kind::mxf4nvf4 with E2M1
+ * elements and E4M3 scales per 16 elements (k = 64).  *flops (host pointer) receives the floating-point operations the
+ * launch performs on the whole device, 2 x 128 x 256 x k per MMA; time the stream around the call to get a rate.
+ * workspace: at least the 256-byte header (the status word records a wait that expired).
+ */
+latmix_status_t latmix_tensor_pipe_probe(int kind, int64_t mma_per_cta, double* flops, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream);
+
+/* Zero the header of a workspace: the status word and the wait limit (enqueued on the stream).  Call once after allocating it. */
 latmix_status_t latmix_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Every wait inside a kernel (on a copy, on the tensor core, on another CTA of a cluster) gives up after about one
+ * second, records LATMIX_ERR_TIMEOUT in the status word and lets the kernel end.  This call replaces that limit, for
+ * kernels launched with this workspace, by `cycles` SM clock cycles (0 = back to the default; values below 32768 act as
+ * 32768).  Enqueued on the stream.  Meant for tests of the failure path and for callers with a tighter deadline.
+ */
+latmix_status_t latmix_workspace_set_wait_limit(void* workspace, size_t workspace_bytes, uint32_t cycles, void* cuda_stream);
 
 /* Synchronise the stream and return the status word of `workspace` (LATMIX_OK if no kernel recorded a problem). */
 latmix_status_t latmix_device_status(void* workspace, void* cuda_stream);

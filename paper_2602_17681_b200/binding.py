@@ -25,6 +25,7 @@ F32, BF16 = 0, 1
 SF_LINEAR, SF_TCGEN05 = 0, 1
 OP_FOLD_WEIGHTS, OP_QUANTIZE_MX, OP_LINEAR, OP_MX_GEMM, OP_FOLD_TWO_SIDED, OP_TRANSFORMATION_MSE = 0, 1, 2, 3, 4, 5
 FLAG_NONE, FLAG_CHECK_FINITE, FLAG_FORCE_SIMT, FLAG_BLOCK_DIAG = 0, 1, 2, 4
+FLAG_TEST_DROP_LOAD = 1 << 16
 FORMATS = {"mxfp4": MXFP4, "mxfp8": MXFP8, "mxint8": MXINT8, "mxint4": MXINT4}
 
 _vp, _i64, _sz, _u32, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_int
@@ -45,7 +46,9 @@ EXPORTS = {
     "latmix_linear": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _i64, _vp, _sz, _u32, _vp]),
     "latmix_linear_static": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _i64, _u32,
                                     ctypes.POINTER(ctypes.c_int), _vp]),
+    "latmix_tensor_pipe_probe": (_int, [_int, _i64, ctypes.POINTER(ctypes.c_double), _vp, _sz, _vp]),
     "latmix_workspace_init": (_int, [_vp, _sz, _vp]),
+    "latmix_workspace_set_wait_limit": (_int, [_vp, _sz, _u32, _vp]),
     "latmix_device_status": (_int, [_vp, _vp]),
 }
 for _name, (_res, _args) in EXPORTS.items():
@@ -116,6 +119,14 @@ def new_workspace(op, M, K, N, fmt, device="cuda"):
     ws = torch.empty(workspace_bytes(op, M, K, N, fmt), dtype=torch.uint8, device=device)
     _check(_lib.latmix_workspace_init(_ptr(ws), ws.numel(), _stream()), "latmix_workspace_init")
     return ws
+
+
+def workspace_init(ws):
+    _check(_lib.latmix_workspace_init(_ptr(ws), ws.numel(), _stream()), "latmix_workspace_init")
+
+
+def workspace_set_wait_limit(ws, cycles):
+    _check(_lib.latmix_workspace_set_wait_limit(_ptr(ws), ws.numel(), cycles, _stream()), "latmix_workspace_set_wait_limit")
 
 
 def device_status(ws):
@@ -195,6 +206,22 @@ def linear(X, A, b, Wq_codes, Wq_scales, c, N, fmt, out=None, ws=None, flags=0):
     return out
 
 
+PIPE_KINDS = {"bf16": 0, "mxf8": 1, "mxf4": 2, "nvf4": 3}
+
+
+def tensor_pipe_probe(kind, ws, mma_per_cta=28672):
+    """TFLOP/s of back-to-back MMAs of the given kind on every SM (latmix_tensor_pipe_probe timed with two events)."""
+    flops = ctypes.c_double()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    _check(_lib.latmix_tensor_pipe_probe(PIPE_KINDS[kind], mma_per_cta, ctypes.byref(flops), _ptr(ws), ws.numel(), _stream()),
+           "latmix_tensor_pipe_probe")
+    ev1.record()
+    ev1.synchronize()
+    _check(device_status(ws), "latmix_tensor_pipe_probe (device status)")
+    return flops.value / (ev0.elapsed_time(ev1) * 1e-3) / 1e12
+
+
 STATIC_SCRATCH_BYTES = 256 + (16 << 20)     # LATMIX_STATIC_SCRATCH_BYTES of include/latmix.h
 
 
@@ -212,17 +239,3 @@ def linear_static(X, A, b, Wq_codes, Wq_scales, c, N, fmt, out, flags=0, wait=Tr
                                      ctypes.byref(dev_status) if wait else None, _stream()), "latmix_linear_static")
     _check(dev_status.value, "latmix_linear_static (device status)")
     return out
-
-
-def scales_to_linear(scales, rows, K, sf):
-    """Host helper for tests: gather the E8M0 bytes of a scale buffer into a [rows, K/32] uint8 array."""
-    import numpy as np
-    buf = scales.cpu().numpy()
-    if sf == SF_LINEAR:
-        return buf[: rows * (K // 32)].reshape(rows, K // 32).copy()
-    r = np.arange(rows)[:, None]
-    kb = np.arange(K // 32)[None, :]
-    kt = ((K // 32 + 7) // 8) * 2
-    off = ((r >> 7) * kt + (kb >> 2)) * 512 + (r & 31) * 16 + ((r >> 5) & 3) * 4 + (kb & 3)
-    assert off[-1, -1] == scale_offset(rows - 1, K // 32 - 1, rows, K, sf)
-    return buf[off]

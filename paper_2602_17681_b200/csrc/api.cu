@@ -46,9 +46,9 @@ static void mx_sizes(int64_t rows, int64_t K, int fmt, int sf, size_t* code_byte
     else *scale_bytes = (size_t)((rows + 127) / 128) * (size_t)sf_k_tiles(K) * 512;
 }
 
-static bool scales_have_padding(int64_t rows, int64_t K, int sf) {
-    return sf == LATMIX_SF_TCGEN05 && (rows % 128 != 0 || (K / 32) % 8 != 0);
-}
+// Padding BLOCKS of the tiled scale layout (K/32 not a multiple of 8) are zeroed before the quantiser runs.  Padding ROWS
+// are not: whatever they hold scales accumulator rows (or columns) that lie outside the result and are never stored.
+static bool scales_have_block_padding(int64_t K, int sf) { return sf == LATMIX_SF_TCGEN05 && (K / 32) % 8 != 0; }
 
 }  // namespace latmix
 
@@ -138,6 +138,16 @@ latmix_status_t latmix_workspace_init(void* workspace, size_t workspace_bytes, v
     return LATMIX_OK;
 }
 
+latmix_status_t latmix_workspace_set_wait_limit(void* workspace, size_t workspace_bytes, uint32_t cycles, void* cuda_stream) {
+    if (workspace == nullptr || workspace_bytes < kWorkspaceHeaderBytes) return LATMIX_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return LATMIX_ERR_INVALID_ARG;
+    // word 1 of the header; the source is pageable host memory, which the runtime has read by the time the call returns
+    if (cudaMemcpyAsync(static_cast<uint32_t*>(workspace) + 1, &cycles, sizeof(cycles), cudaMemcpyHostToDevice,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return LATMIX_ERR_CUDA;
+    return LATMIX_OK;
+}
+
 latmix_status_t latmix_device_status(void* workspace, void* cuda_stream) {
     if (workspace == nullptr) return LATMIX_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -164,7 +174,7 @@ latmix_status_t latmix_quantize_mx(const void* X, latmix_dtype_t x_dtype, const 
     if ((s = check_device()) != LATMIX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint32_t* status = static_cast<uint32_t*>(workspace);
-    if (scales_have_padding(M, K, sf)) {
+    if (scales_have_block_padding(K, sf)) {
         size_t cb, sb;
         mx_sizes(M, K, fmt, sf, &cb, &sb);
         if (cudaMemsetAsync(scales, 0, sb, st) != cudaSuccess) return LATMIX_ERR_CUDA;
@@ -242,7 +252,7 @@ latmix_status_t latmix_fold_weights(const void* A_inv, const float* b, const voi
     if (N == 0 || K == 0) return LATMIX_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* base = static_cast<uint8_t*>(workspace);
-    if (scales_have_padding(N, K, sf)) {
+    if (scales_have_block_padding(K, sf)) {
         size_t cb, sb;
         mx_sizes(N, K, fmt, sf, &cb, &sb);
         if (cudaMemsetAsync(Wq_scales, 0, sb, st) != cudaSuccess) return LATMIX_ERR_CUDA;
@@ -291,7 +301,7 @@ latmix_status_t latmix_fold_weights_two_sided(const float* A_in_inv, const float
     uint32_t* status = static_cast<uint32_t*>(workspace);
     uint8_t* codes = static_cast<uint8_t*>(Wq_codes);
     uint8_t* scales = static_cast<uint8_t*>(Wq_scales);
-    if (scales_have_padding(N, K, sf)) {
+    if (scales_have_block_padding(K, sf)) {
         size_t cb, sb;
         mx_sizes(N, K, fmt, sf, &cb, &sb);
         if (cudaMemsetAsync(Wq_scales, 0, sb, st) != cudaSuccess) return LATMIX_ERR_CUDA;

@@ -1,6 +1,7 @@
 // sm_100a building blocks for the tensor-core kernels: mbarrier, TMA (cp.async.bulk[.tensor]), tensor memory
 // (tcgen05.alloc/ld/cp), tcgen05.mma descriptors and issue, all as thin inline-PTX wrappers.
-// Every wait is bounded: after kWaitLimitCycles it gives up, records LATMIX_ERR_TIMEOUT and returns false.
+// Every wait is bounded: after kWaitLimitCycles (or the limit the workspace header carries, see wait_limit_cycles) it gives
+// up, records LATMIX_ERR_TIMEOUT and returns false.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -39,12 +40,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Word 1 of the workspace header, when not zero, replaces kWaitLimitCycles (latmix_workspace_set_wait_limit).  It is read
+// only by waits that have already lasted kWaitCheckCycles, so an ordinary wait never touches global memory.
+constexpr long long kWaitCheckCycles = 1ll << 15;
+__device__ __forceinline__ bool wait_expired(long long waited, const uint32_t* status) {
+    if (waited <= kWaitCheckCycles) return false;
+    const uint32_t v = *reinterpret_cast<const volatile uint32_t*>(status + 1);
+    return waited > (v != 0u ? (long long)v : kWaitLimitCycles);
+}
+
 // Bounded wait for the phase with the given parity to complete.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (wait_expired(clock64() - t0, status)) {
             atomicOr(status, 1u << LATMIX_ERR_TIMEOUT);
             return false;
         }
@@ -60,7 +70,7 @@ __device__ __forceinline__ void mbar_wait_or_flag(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if ((*reinterpret_cast<volatile uint32_t*>(status) & (1u << LATMIX_ERR_TIMEOUT)) || clock64() - t0 > kWaitLimitCycles) {
+        if ((*reinterpret_cast<volatile uint32_t*>(status) & (1u << LATMIX_ERR_TIMEOUT)) || wait_expired(clock64() - t0, status)) {
             atomicOr(status, 1u << LATMIX_ERR_TIMEOUT);
             return;
         }
@@ -281,6 +291,9 @@ LATMIX_MMA_BLOCK_SCALED(mma_mxf4_lean, "tcgen05.mma.cta_group::1.kind::mxf4.bloc
 LATMIX_MMA_BLOCK_SCALED(mma_mxf8_lean, "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.scale_vec::1X")
 LATMIX_MMA_BLOCK_SCALED(mma_mxf4_pair_lean, "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X")
 LATMIX_MMA_BLOCK_SCALED(mma_mxf8_pair_lean, "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X")
+// NVFP4: E2M1 elements, one UE4M3 scale per 16 elements (four per row and MMA, all four bytes of a scale column)
+LATMIX_MMA_BLOCK_SCALED(mma_nvf4_lean, "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X")
+LATMIX_MMA_BLOCK_SCALED(mma_nvf4_pair_lean, "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X")
 #undef LATMIX_MMA_BLOCK_SCALED
 
 // Dense bf16 x bf16 -> fp32; the B descriptor's low word also carries its leading byte offset (bits 16-29).

@@ -99,23 +99,6 @@ def make_transform(K, seed, a_dtype="bf16", b_std=0.1, device="cpu"):
     return A, b, A_inv
 
 
-def make_block_diag_transform(K, seed, block=32, a_dtype="bf16", b_std=0.1, device="cpu"):
-    """Cheap A for very wide layers: independent Haar blocks of size `block` on
-    the diagonal times diag(s).  Same (A, b, A_inv) contract as make_transform."""
-    g = _gen(seed * 7919 + 5, device)
-    nb = K // block
-    G = torch.randn(nb, block, block, generator=g, device=device, dtype=torch.float64)
-    Q, R = torch.linalg.qr(G)
-    Q = Q * torch.sign(torch.diagonal(R, dim1=1, dim2=2))[:, None, :]
-    s = torch.exp(torch.empty(K, device=device, dtype=torch.float64).uniform_(
-        math.log(0.5), math.log(2.0), generator=g))
-    A = torch.block_diag(*Q) * s[None, :]
-    A = _storage(A, a_dtype)
-    b = (torch.randn(K, generator=g, device=device, dtype=torch.float64) * b_std).float()
-    A_inv = torch.linalg.inv(A.double()).float().contiguous()
-    return A, b, A_inv
-
-
 def make_block_transform(K, seed, kind="haar", block=32, a_dtype="bf16", b_std=0.0, device="cpu"):
     """Block-wise online transform as [K/block, block, block] blocks (block i acts on elements i*block ...).
 

@@ -15,6 +15,16 @@ def sf_offsets(rows, K):
     return ((r >> 7) * kt + (kb >> 2)) * 512 + (r & 31) * 16 + ((r >> 5) & 3) * 4 + (kb & 3)
 
 
+def scales_to_linear(B, scales, rows, K, sf):
+    """Gather the scale bytes of a device scale buffer into a [rows, K/32] uint8 array."""
+    buf = scales.cpu().numpy()
+    if sf == B.SF_LINEAR:
+        return buf[: rows * (K // 32)].reshape(rows, K // 32).copy()
+    off = sf_offsets(rows, K)
+    assert off[-1, -1] == B.scale_offset(rows - 1, K // 32 - 1, rows, K, sf)
+    return buf[off]
+
+
 def codes_to_numpy(codes_t, rows, K, fmt):
     buf = codes_t.cpu().numpy()
     if fmt == 0:
@@ -87,3 +97,46 @@ def fma_unit(K):
 def accumulation_tau(X64, A64, unit):
     """Per-element bound on the difference between an fp32-accumulated and the exact product."""
     return unit * (np.abs(X64) @ np.abs(A64)) + 1e-30
+
+
+K_PER_MMA = {"mxfp4": 64, "mxfp8": 32, "mxint4": 32, "mxint8": 16}      # MXINT8 runs as an exact bf16 product
+
+
+def block_scaled_unit(K, fmt_name, simt=False):
+    """Relative size of the accumulation error of the block-scaled product, per unit of sum |dq(a)||dq(w)|.
+
+    Products of element values and power-of-two scales are exact.  On the tensor cores the fp32 accumulator is
+    rounded (or truncated: 2^-23) once per MMA instruction, K / k_per_mma times; a few more roundings cover the sum
+    inside one instruction.  The CUDA-core kernel adds one 32-term fp32 FMA chain per block and then K/32 block sums
+    across 32 lanes and a five-step shuffle tree."""
+    if simt:
+        return (32 + K / 1024.0 + 6.0) * 2.0 ** -24
+    return (K / K_PER_MMA[fmt_name] + 4.0) * 2.0 ** -23
+
+
+def gemm_error_ratio(out, ref, a_codes, a_scales, w_codes, w_scales, fmt_name, c=None):
+    """Largest |out - ref| in units of 2^-24 of sum_k |dq(a)_k| |dq(w)_k| (+ |c|)."""
+    Ad = np.abs(orc.mx_dequantize(a_codes, a_scales, fmt_name))
+    Wd = np.abs(orc.mx_dequantize(w_codes, w_scales, fmt_name))
+    mag = Ad @ Wd.T + (0.0 if c is None else np.abs(np.asarray(c, dtype=np.float64))[None, :])
+    err = np.abs(np.asarray(out, dtype=np.float64) - ref)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ratio = np.where(mag > 0, err / (mag * 2.0 ** -24), np.where(err > 0, np.inf, 0.0))
+    return float(ratio.max()), mag
+
+
+def assert_gemm_parity(out, ref, a_codes, a_scales, w_codes, w_scales, fmt_name, K, c=None, simt=False, tol=1e-4, tag=""):
+    """Block-scaled product against the fp64 contraction of the same codes: relative Frobenius norm within `tol` AND every
+    element within the accumulation bound  |out - ref| <= u (sum_k |dq(a)_k||dq(w)_k| + |c|) + one fp32 rounding of the
+    result (u: block_scaled_unit; simt=None takes the larger of the two kernels' units where the shape decides which one
+    runs).  A single wrong element fails the second check at any matrix size."""
+    out = np.asarray(out, dtype=np.float64)
+    assert np.isfinite(out).all(), tag
+    assert rel_fro(out, ref) < tol, (tag, rel_fro(out, ref))
+    ratio, mag = gemm_error_ratio(out, ref, a_codes, a_scales, w_codes, w_scales, fmt_name, c)
+    unit = (max(block_scaled_unit(K, fmt_name, False), block_scaled_unit(K, fmt_name, True)) if simt is None
+            else block_scaled_unit(K, fmt_name, simt))
+    bound = unit * mag + 2.0 ** -23 * np.abs(ref) + 1e-300
+    bad = np.abs(out - ref) > bound
+    print(f"GEMM_ERR {tag} fmt={fmt_name} K={K} max_err_over_2^-24_mag={ratio:.2f} bound={unit * 2 ** 24:.1f}")
+    assert not bad.any(), (tag, int(bad.sum()), ratio)

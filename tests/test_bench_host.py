@@ -50,3 +50,31 @@ def test_two_gloo_ranks_agree_on_the_slowest_time():
     out = mgr.dict()
     mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
     assert out[0] == out[1] == (15.0, 1001)
+
+
+@pytest.mark.timeout(180)
+def test_gpus_flag_spawns_that_many_ranks():
+    """`bench.py --gpus 2` without a launcher starts two ranks itself (here on gloo, no GPU work) and reports n_gpus = 2;
+    asked for more GPUs than the machine has, the GPU arm refuses instead of running on fewer."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--plumbing-only", "--workload", "cfg1"],
+                       capture_output=True, text=True, env=env, timeout=170)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([ln for ln in r.stdout.splitlines() if ln.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["ms_slowest_rank"] == 2.0 and line["rows_total"] == 2 * 2048
+    if torch.cuda.device_count() < 64:
+        r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "64", "--steps", "1"],
+                           capture_output=True, text=True, env=env, timeout=170)
+        assert r.returncode == 2 and "GPU(s) visible" in r.stderr
+
+
+def test_regime_follows_the_sampled_clock():
+    import bench
+    full = dict(sm_mhz=1965.0, sm_max_mhz=1965.0, reasons=[])
+    capped = dict(sm_mhz=1400.0, sm_max_mhz=1965.0, reasons=["sw_power_cap"])
+    slow = dict(sm_mhz=1400.0, sm_max_mhz=1965.0, reasons=[])
+    assert bench.pick_regime(full, 4.0) == "burst" and bench.pick_regime(full, 2000.0) == "burst"
+    assert bench.pick_regime(capped, 4.0) == "sustained" and bench.pick_regime(slow, 2000.0) == "sustained"
+    assert bench.pick_regime(dict(sm_mhz=None, sm_max_mhz=None, reasons=[]), 2000.0) == "burst"

@@ -38,7 +38,11 @@ def test_static_scratch_matches_workspace_call_twice_in_a_row(B):
         want = B.linear(L["X"], L["A"], L["b"], wq, wsc, c, cfg.N, fmt, ws=ws)
         assert B.device_status(ws) == B.OK
         got = torch.full((cfg.M, cfg.N), float("nan"), dtype=torch.float32, device=dev)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         B.linear_static(L["X"], L["A"], L["b"], wq, wsc, c, cfg.N, fmt, out=got)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before       # the call took no device memory (cudaMemGetInfo)
         assert torch.isfinite(got).all()
         # same kernels, same inputs: the tolerance of the layer tests (relative Frobenius 1e-4) is met with zero
         assert H.rel_fro(got.cpu().numpy(), want.double().cpu().numpy()) <= 1e-4
