@@ -28,6 +28,14 @@ chain (which also fixes the sign of the output-projection bias).
 MXINT8's symmetric clamp (+-127) is this repository's choice: parity unpinned
 beyond the OCP text for that format.  MXINT4 has no published definition at
 all (see the format table below): parity unpinned.
+NVFP4 (appendix "NVFP Quantization Format Evaluation") is evaluated by the
+paper but defined nowhere in it; the functions nvfp4_* follow the vendor's
+public description of the format (blocks of 16, E2M1 elements, an E4M3 block
+scale, one fp32 scale per tensor).  Their conversions are pinned (NVIDIA's host
+E4M3 / E2M1 routines, an exact-rational brute force with explicit fp32
+roundings, the reduction to E2M1 rounding when the scale is a power of two);
+the recipe that picks the block scale (amax / 6 over the tensor scale, rounded
+to nearest) is a reading: parity unpinned for that choice.
 """
 from __future__ import annotations
 
@@ -232,6 +240,110 @@ def unpack_fp4(packed):
     out[..., 0::2] = packed & 0xF
     out[..., 1::2] = packed >> 4
     return out
+
+
+# --------------------------------------------------------------------------
+# NVFP4 (appendix "NVFP Quantization Format Evaluation"; the format itself is
+# the vendor's: blocks of 16, E2M1 elements, E4M3 block scale, fp32 tensor scale)
+# --------------------------------------------------------------------------
+NVFP4_BLOCK = 16
+
+
+def nvfp4_quantize(Y, tensor_scale, block=NVFP4_BLOCK):
+    """x ~ e * d * g with e an E2M1 element, d the block's E4M3 scale and g the tensor's fp32 scale (an input).
+
+    Unlike the power-of-two MX scale, d * g is not a power of two, so the precision of the division decides codes.
+    The format's arithmetic is taken to be fp32, round to nearest even, in this order (each step one IEEE operation):
+        y    = fp32(Y)                          the values are fp32 numbers when they reach the quantiser
+        t    = (amax / 6) / g                   two divisions; 6 = largest E2M1 magnitude
+        d    = E4M3(t)                          round to nearest even, saturate at 448, positive
+        s    = d * g                            the decode scale of the block
+        r    = 1 / s   (0 when s == 0)
+        e_j  = E2M1(y_j * r)                    round to nearest even, saturate at 6, sign bit kept
+    Returns (codes uint8 [rows, K], scale codes uint8 [rows, K / block])."""
+    f32 = np.float32
+    Y = np.asarray(Y, dtype=np.float64)
+    assert Y.ndim == 2 and Y.shape[1] % block == 0 and np.all(np.isfinite(Y))
+    g = f32(tensor_scale)
+    assert np.isfinite(g) and g > 0
+    rows, K = Y.shape
+    y = Y.astype(f32).reshape(rows, K // block, block)
+    amax = np.abs(y).max(axis=2)
+    with np.errstate(over="ignore", under="ignore", divide="ignore"):
+        t = (amax / f32(6.0)) / g
+        t = np.minimum(t, f32(3.0e38))                        # an overflow to infinity saturates like any large value
+        d_code = quantize_elements_arith(t.astype(np.float64), MXFP8)
+        d = decode_elements(d_code, MXFP8).astype(f32)       # exact: E4M3 values are fp32 numbers
+        s = d * g
+        r = np.where(s > 0, f32(1.0) / np.where(s > 0, s, f32(1.0)), f32(0.0)).astype(f32)
+        v = y * r[:, :, None]
+        v = np.clip(v, f32(-3.0e38), f32(3.0e38))
+    codes = quantize_elements_arith(v.astype(np.float64), MXFP4).reshape(rows, K)
+    return codes, d_code.astype(np.uint8)
+
+
+def nvfp4_dequantize(codes, scale_codes, tensor_scale, block=NVFP4_BLOCK):
+    """The real numbers the codes stand for: element value * E4M3 block scale * tensor scale (exact in fp64)."""
+    rows, K = codes.shape
+    vals = decode_elements(codes, MXFP4).reshape(rows, K // block, block)
+    d = decode_elements(scale_codes, MXFP8)
+    return (vals * d[:, :, None]).reshape(rows, K) * float(np.float32(tensor_scale))
+
+
+def nvfp4_matmul(a_codes, a_scales, g_a, w_codes, w_scales, g_w, c, block=NVFP4_BLOCK):
+    """out = dq(Qa) dq(Qw)^T + c in fp64 (Qw stored N x K)."""
+    out = nvfp4_dequantize(a_codes, a_scales, g_a, block) @ nvfp4_dequantize(w_codes, w_scales, g_w, block).T
+    if c is not None:
+        out = out + np.asarray(c, dtype=np.float64)[None, :]
+    return out
+
+
+def nvfp4_tensor_scale(amax_tensor):
+    """The tensor scale that maps the tensor's largest magnitude onto the largest block scale times the largest
+    element: g = amax / (448 * 6), in fp32 (the vendor's recipe; any positive fp32 number is a valid g)."""
+    g = np.float32(amax_tensor) / np.float32(448.0 * 6.0)
+    return np.float32(g) if g > 0 else np.float32(1.0)
+
+
+def nvfp4_quantize_block_exact(values, tensor_scale, block=NVFP4_BLOCK):
+    """One NVFP4 block with rational arithmetic and explicit roundings to fp32 / E4M3 / E2M1 done on integers: no
+    floating-point operation decides anything.  For brute-force pins on tiny inputs."""
+    from fractions import Fraction
+
+    def round_to_precision(x, man_bits, e_min, x_max):
+        """Nearest number with `man_bits` explicit mantissa bits and smallest normal exponent e_min (subnormals below
+        it), ties to even, saturating at x_max; x >= 0 a Fraction."""
+        if x == 0:
+            return Fraction(0)
+        e = 0
+        while Fraction(2) ** (e + 1) <= x:
+            e += 1
+        while Fraction(2) ** e > x:
+            e -= 1
+        e = max(e, e_min)
+        ulp = Fraction(2) ** (e - man_bits)
+        q, rem = divmod(x, ulp)
+        if rem * 2 > ulp or (rem * 2 == ulp and q % 2 == 1):
+            q += 1
+        return min(q * ulp, x_max)
+
+    f32_max = Fraction(2) ** 128 - Fraction(2) ** 104
+    f32 = lambda x: round_to_precision(x, 23, -126, f32_max)
+    g = Fraction(float(np.float32(tensor_scale)))
+    vals = [Fraction(float(np.float32(x))) for x in values]
+    amax = max(abs(x) for x in vals)
+    t = f32(f32(amax / 6) / g)
+    d = round_to_precision(t, 3, -6, Fraction(448))
+    s = f32(d * g)
+    r = f32(1 / s) if s > 0 else Fraction(0)
+    grid = [Fraction(float(x)) for x in MXFP4.grid]
+    codes = []
+    for x, xf in zip(vals, values):
+        z = f32(abs(x) * r)
+        best = min(range(len(grid)), key=lambda i: (abs(z - grid[i]), i % 2, i))
+        codes.append(best | (int(bool(np.signbit(np.float32(xf)))) << 3))
+    e4m3 = [Fraction(float(x)) for x in MXFP8.grid]
+    return codes, e4m3.index(d)
 
 
 # --------------------------------------------------------------------------

@@ -70,7 +70,9 @@ def test_stale_scale_padding_rows_do_not_reach_the_output(B):
 
 def test_tensor_pipe_probe_runs(B):
     ws = B.new_workspace(B.OP_QUANTIZE_MX, 0, 64, 0, 0)
-    rates = {k: B.tensor_pipe_probe(k, ws, mma_per_cta=4096) for k in ("bf16", "mxf8", "mxf4", "nvf4")}
+    for k in ("bf16", "mxf8", "mxf4", "nvf4"):            # first launches carry module loading
+        B.tensor_pipe_probe(k, ws, mma_per_cta=64)
+    rates = {k: max(B.tensor_pipe_probe(k, ws) for _ in range(3)) for k in ("bf16", "mxf8", "mxf4", "nvf4")}
     assert B.device_status(ws) == B.OK
     # the pipes' nominal ratios 1 : 2 : 4 : 4, loosely (clocks move between launches)
     assert 1.5 < rates["mxf8"] / rates["bf16"] < 2.5 and 3.0 < rates["mxf4"] / rates["bf16"] < 5.0, rates
