@@ -572,7 +572,7 @@ def run_mma_peak(args, local_rank):
     dev = torch.device("cuda", local_rank)
     peaks = load_peaks()
     ws = B.new_workspace(B.OP_QUANTIZE_MX, 0, 64, 0, B.MXFP4, dev)
-    nominal = {"bf16": 1.0, "mxf8": 2.0, "mxf4": 4.0, "nvf4": 4.0}
+    nominal = {"bf16": 1.0, "mxf8": 2.0, "mxf4": 4.0, "nvf4": 4.0, "mxf4_pair": 4.0}
     for kind in nominal:                                   # warm-up
         B.tensor_pipe_probe(kind, ws=ws)
     sampler = ClockSampler(local_rank)

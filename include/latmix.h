@@ -62,7 +62,18 @@ typedef enum {
      * (symmetric 4-bit range), value = k, r_max 2, round to nearest even, |k| = 8 saturates to 7.  Each element is STORED
      * as one byte holding the E4M3 encoding of k (zero always as +0): the 8-bit block-scaled tensor-core kind then consumes
      * the codes unchanged and every product stays exact; buffer sizes and the GEMM are those of LATMIX_MXFP8_E4M3. */
-    LATMIX_MXINT4 = 3
+    LATMIX_MXINT4 = 3,
+    /* NVFP4, which the paper evaluates in its appendix "NVFP Quantization Format Evaluation" without defining it; taken from
+     * the vendor's public description: E2M1 elements packed like MXFP4, blocks of 16 (not 32) along K, one E4M3 scale byte
+     * per block (positive, finite), and one fp32 scale g per tensor:  x ~ element * block scale * g.  The caller chooses g
+     * (commonly max|x| / (448 * 6)) and stores it as an fp32 number in the 16-byte trailer at the end of the scale buffer
+     * (latmix_tensor_scale_offset) BEFORE the quantising call; the calls that consume the buffer read it from there.
+     * Quantisation, in fp32, one correctly rounded operation per step: t = (amax / 6) / g; d = E4M3(t) (nearest even,
+     * saturating); s = d * g; r = 1 / s (0 if s = 0); code = E2M1(x * r) (nearest even, saturating, sign kept).
+     * g must be a normal fp32 number in [2^-96, 2^96].  K must be a multiple of 64.  The choice of d is a reading of the
+     * vendor's recipe.  Supported by latmix_quantize_mx (not with LATMIX_FLAG_BLOCK_DIAG), latmix_fold_weights,
+     * latmix_mx_gemm and latmix_linear; the other calls return LATMIX_ERR_UNSUPPORTED. */
+    LATMIX_NVFP4 = 4
 } latmix_format_t;
 
 typedef enum { LATMIX_F32 = 0, LATMIX_BF16 = 1 } latmix_dtype_t;
@@ -102,7 +113,8 @@ enum {
 /* Bits 8-11 of `flags` select a kernel where several apply (for tests and measurements; results agree bit for bit in the
  * block-scaled product, up to near-ties in the transform): 0 = the library's choice by shape, 1-3 = single-CTA tensor-core
  * kernels (tile 128 x 128, 128 x 192, 128 x 256), 4 = the small-batch kernels (product and transform: M <= 64,
- * transform K <= 16384), 8 = the CTA-pair kernels.  A value whose kernel does not take the shape falls back to the next that does. */
+ * transform K <= 16384), 8 = the CTA-pair kernels (product: 256 x 192 tiles), 9 = the product on CTA pairs with 256 x 256
+ * tiles (the default for M > 128).  A value whose kernel does not take the shape falls back to the next that does. */
 #define LATMIX_FLAG_KERNEL(v) ((uint32_t)(v) << 8)
 
 /* Host helpers (no device work). ------------------------------------------------------------------------- */
@@ -113,6 +125,14 @@ latmix_status_t latmix_mx_sizes(int64_t rows, int64_t K, latmix_format_t fmt, la
 
 /* Byte offset of the scale of (row, kblock) in a scale buffer with the given layout; (size_t)-1 on bad input. */
 size_t latmix_scale_offset(int64_t row, int64_t kblock, int64_t rows, int64_t K, latmix_sf_layout_t sf);
+
+/* The same for any format: for LATMIX_NVFP4 `kblock` counts blocks of 16 elements (K/16 per row, tiles of 128 rows x 4
+ * blocks, blocks padded to a multiple of 16); for the MX formats it is latmix_scale_offset. */
+size_t latmix_scale_offset_fmt(int64_t row, int64_t kblock, int64_t rows, int64_t K, latmix_format_t fmt, latmix_sf_layout_t sf);
+
+/* LATMIX_NVFP4: byte offset, inside a scale buffer of latmix_mx_sizes(rows, K, LATMIX_NVFP4, sf) bytes, of the fp32 tensor
+ * scale (the start of the 16-byte trailer behind the block scales); (size_t)-1 for the other formats. */
+size_t latmix_tensor_scale_offset(int64_t rows, int64_t K, latmix_format_t fmt, latmix_sf_layout_t sf);
 
 /* Bytes of device workspace the given call needs for these sizes (always >= 256: the status word lives there). */
 latmix_status_t latmix_workspace_bytes(latmix_op_t op, int64_t M, int64_t K, int64_t N, latmix_format_t fmt,
@@ -264,7 +284,9 @@ latmix_status_t latmix_linear_static(const void* X, latmix_dtype_t x_dtype, cons
  * multiple of 4; 4 .. 2^22) tcgen05.mma of shape 128 x 256 x k back to back on operands that sit in shared memory; the
  * results are discarded.  kind: 0 = kind::f16 with bf16 operands (k = 16), 1 = kind::mxf8f6f4 with E4M3 elements and E8M0
  * block scales (k = 32), 2 = kind::mxf4 with E2M1 elements and E8M0 block scales (k = 64), 3 = kind::mxf4nvf4 with E2M1
- * elements and E4M3 scales per 16 elements (k = 64).  *flops (host pointer) receives the floating-point operations the
+ * elements and E4M3 scales per 16 elements (k = 64), 4 = kind::mxf4 again but issued by CTA pairs (cta_group::2, one 256 x 256 x
+ * 64 MMA per step and pair, `mma_per_cta` steps per pair; bits 8-23 of `kind`, a multiple of 4 or 0, make the issuing thread add
+ * a tcgen05.commit after every so many MMAs, as a pipelined kernel does to release its stages).  *flops (host pointer) receives the floating-point operations the
  * launch performs on the whole device, 2 x 128 x 256 x k per MMA; time the stream around the call to get a rate.
  * workspace: at least the 256-byte header (the status word records a wait that expired).
  */
@@ -281,6 +303,13 @@ latmix_status_t latmix_workspace_init(void* workspace, size_t workspace_bytes, v
  * 32768).  Enqueued on the stream.  Meant for tests of the failure path and for callers with a tighter deadline.
  */
 latmix_status_t latmix_workspace_set_wait_limit(void* workspace, size_t workspace_bytes, uint32_t cycles, void* cuda_stream);
+
+/*
+ * LATMIX_NVFP4 with latmix_linear: the activation codes and scales live in the workspace, so the activations' tensor scale
+ * cannot be written into their trailer by the caller; this call stores it in the workspace header (enqueued on the stream),
+ * and latmix_linear moves it to the trailer on every call.  It stays until the header is re-initialised.  Must be positive.
+ */
+latmix_status_t latmix_workspace_set_tensor_scale(void* workspace, size_t workspace_bytes, float tensor_scale, void* cuda_stream);
 
 /* Synchronise the stream and return the status word of `workspace` (LATMIX_OK if no kernel recorded a problem). */
 latmix_status_t latmix_device_status(void* workspace, void* cuda_stream);

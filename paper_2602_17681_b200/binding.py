@@ -20,13 +20,13 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 # enums of include/latmix.h
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE = range(8)
-MXFP4, MXFP8, MXINT8, MXINT4 = 0, 1, 2, 3
+MXFP4, MXFP8, MXINT8, MXINT4, NVFP4 = 0, 1, 2, 3, 4
 F32, BF16 = 0, 1
 SF_LINEAR, SF_TCGEN05 = 0, 1
 OP_FOLD_WEIGHTS, OP_QUANTIZE_MX, OP_LINEAR, OP_MX_GEMM, OP_FOLD_TWO_SIDED, OP_TRANSFORMATION_MSE = 0, 1, 2, 3, 4, 5
 FLAG_NONE, FLAG_CHECK_FINITE, FLAG_FORCE_SIMT, FLAG_BLOCK_DIAG = 0, 1, 2, 4
 FLAG_TEST_DROP_LOAD = 1 << 16
-FORMATS = {"mxfp4": MXFP4, "mxfp8": MXFP8, "mxint8": MXINT8, "mxint4": MXINT4}
+FORMATS = {"mxfp4": MXFP4, "mxfp8": MXFP8, "mxint8": MXINT8, "mxint4": MXINT4, "nvfp4": NVFP4}
 
 _vp, _i64, _sz, _u32, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_int
 _szp = ctypes.POINTER(ctypes.c_size_t)
@@ -34,6 +34,9 @@ _szp = ctypes.POINTER(ctypes.c_size_t)
 EXPORTS = {
     "latmix_mx_sizes": (_int, [_i64, _i64, _int, _int, _szp, _szp]),
     "latmix_scale_offset": (_sz, [_i64, _i64, _i64, _i64, _int]),
+    "latmix_scale_offset_fmt": (_sz, [_i64, _i64, _i64, _i64, _int, _int]),
+    "latmix_tensor_scale_offset": (_sz, [_i64, _i64, _int, _int]),
+    "latmix_workspace_set_tensor_scale": (_int, [_vp, _sz, ctypes.c_float, _vp]),
     "latmix_workspace_bytes": (_int, [_int, _i64, _i64, _i64, _int, _szp]),
     "latmix_status_string": (ctypes.c_char_p, [_int]),
     "latmix_launch_count": (ctypes.c_uint64, []),
@@ -104,6 +107,25 @@ def scale_offset(row, kblock, rows, K, sf=SF_TCGEN05):
     return _lib.latmix_scale_offset(row, kblock, rows, K, sf)
 
 
+def scale_offset_fmt(row, kblock, rows, K, fmt, sf=SF_TCGEN05):
+    return _lib.latmix_scale_offset_fmt(row, kblock, rows, K, fmt, sf)
+
+
+def tensor_scale_offset(rows, K, fmt, sf=SF_TCGEN05):
+    return _lib.latmix_tensor_scale_offset(rows, K, fmt, sf)
+
+
+def set_tensor_scale(scales, rows, K, fmt, sf, value):
+    """NVFP4: write the tensor's fp32 scale into the trailer of a scale buffer (a device-side copy on the current stream)."""
+    off = tensor_scale_offset(rows, K, fmt, sf)
+    assert off != ctypes.c_size_t(-1).value
+    scales[off:off + 4].view(torch.float32).fill_(float(value))
+
+
+def workspace_set_tensor_scale(ws, value):
+    _check(_lib.latmix_workspace_set_tensor_scale(_ptr(ws), ws.numel(), float(value), _stream()), "latmix_workspace_set_tensor_scale")
+
+
 def workspace_bytes(op, M, K, N, fmt):
     n = ctypes.c_size_t()
     _check(_lib.latmix_workspace_bytes(op, M, K, N, fmt, ctypes.byref(n)), "latmix_workspace_bytes")
@@ -139,10 +161,13 @@ def alloc_mx(rows, K, fmt, sf=SF_TCGEN05, device="cuda"):
             torch.empty(max(sb, 16), dtype=torch.uint8, device=device))
 
 
-def fold_weights(A_inv, b, W, bias, fmt, sf=SF_TCGEN05, dump=False, ws=None, flags=0):
-    """-> (Wq_codes, Wq_scales, c, W~^T dump or None).  W is K x N; codes are N x K (K-major)."""
+def fold_weights(A_inv, b, W, bias, fmt, sf=SF_TCGEN05, dump=False, ws=None, flags=0, tensor_scale=None):
+    """-> (Wq_codes, Wq_scales, c, W~^T dump or None).  W is K x N; codes are N x K (K-major).  NVFP4: tensor_scale is
+    written into the new scale buffer's trailer before the call."""
     K, N = W.shape
     codes, scales = alloc_mx(N, K, fmt, sf, W.device)
+    if tensor_scale is not None:
+        set_tensor_scale(scales, N, K, fmt, sf, tensor_scale)
     c = torch.empty(N, dtype=torch.float32, device=W.device)
     dumped = torch.empty(N, K, dtype=torch.float32, device=W.device) if dump else None
     ws = new_workspace(OP_FOLD_WEIGHTS, 0, K, N, fmt, W.device) if ws is None else ws
@@ -165,10 +190,13 @@ def fold_weights_two_sided(A_in_inv, b_in, W, bias, A_out, v_out, fmt, sf=SF_TCG
     return codes, scales, c, dumped
 
 
-def quantize_mx(X, A, b, fmt, sf=SF_TCGEN05, dump=False, ws=None, flags=0, out=None):
-    """-> (codes, scales, Y dump or None) = Q(X A + b); A None = identity."""
+def quantize_mx(X, A, b, fmt, sf=SF_TCGEN05, dump=False, ws=None, flags=0, out=None, tensor_scale=None):
+    """-> (codes, scales, Y dump or None) = Q(X A + b); A None = identity.  NVFP4: tensor_scale is written into the scale
+    buffer's trailer before the call (leave it None if the buffer passed in `out` already carries it)."""
     M, K = X.shape
     codes, scales = alloc_mx(M, K, fmt, sf, X.device) if out is None else out
+    if tensor_scale is not None:
+        set_tensor_scale(scales, M, K, fmt, sf, tensor_scale)
     dumped = torch.empty(M, K, dtype=torch.float32, device=X.device) if dump else None
     ws = new_workspace(OP_QUANTIZE_MX, M, K, 0, fmt, X.device) if ws is None else ws
     _check(_lib.latmix_quantize_mx(_ptr(X), _dtype(X), _ptr(A), _ptr(b), M, K, fmt, sf, _ptr(codes), _ptr(scales),
@@ -206,15 +234,15 @@ def linear(X, A, b, Wq_codes, Wq_scales, c, N, fmt, out=None, ws=None, flags=0):
     return out
 
 
-PIPE_KINDS = {"bf16": 0, "mxf8": 1, "mxf4": 2, "nvf4": 3}
+PIPE_KINDS = {"bf16": 0, "mxf8": 1, "mxf4": 2, "nvf4": 3, "mxf4_pair": 4}
 
 
-def tensor_pipe_probe(kind, ws, mma_per_cta=28672):
+def tensor_pipe_probe(kind, ws, mma_per_cta=28672, commit_every=0):
     """TFLOP/s of back-to-back MMAs of the given kind on every SM (latmix_tensor_pipe_probe timed with two events)."""
     flops = ctypes.c_double()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    _check(_lib.latmix_tensor_pipe_probe(PIPE_KINDS[kind], mma_per_cta, ctypes.byref(flops), _ptr(ws), ws.numel(), _stream()),
+    _check(_lib.latmix_tensor_pipe_probe(PIPE_KINDS[kind] | (commit_every << 8), mma_per_cta, ctypes.byref(flops), _ptr(ws), ws.numel(), _stream()),
            "latmix_tensor_pipe_probe")
     ev1.record()
     ev1.synchronize()

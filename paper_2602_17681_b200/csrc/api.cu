@@ -13,7 +13,10 @@ void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_r
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-static inline bool valid_fmt(int f) { return f == LATMIX_MXFP4_E2M1 || f == LATMIX_MXFP8_E4M3 || f == LATMIX_MXINT8 || f == LATMIX_MXINT4; }
+static inline bool valid_fmt(int f) {
+    return f == LATMIX_MXFP4_E2M1 || f == LATMIX_MXFP8_E4M3 || f == LATMIX_MXINT8 || f == LATMIX_MXINT4 || f == LATMIX_NVFP4;
+}
+static inline bool packs_two_codes(int f) { return f == LATMIX_MXFP4_E2M1 || f == LATMIX_NVFP4; }
 static inline bool valid_dtype(int d) { return d == LATMIX_F32 || d == LATMIX_BF16; }
 static inline bool valid_sf(int s) { return s == LATMIX_SF_LINEAR || s == LATMIX_SF_TCGEN05; }
 
@@ -36,19 +39,31 @@ static latmix_status_t check_device() {
 static latmix_status_t shape_check(int64_t rows, int64_t K, int fmt) {
     if (rows < 0 || K < 0) return LATMIX_ERR_INVALID_ARG;
     if (K % 32 != 0) return LATMIX_ERR_SHAPE;
-    if (fmt == LATMIX_MXFP4_E2M1 && K % 64 != 0) return LATMIX_ERR_SHAPE;
+    if (packs_two_codes(fmt) && K % 64 != 0) return LATMIX_ERR_SHAPE;
     return LATMIX_OK;
 }
 
+constexpr size_t kTensorScaleTrailerBytes = 16;     // NVFP4: the tensor's fp32 scale sits behind the block scales
+
 static void mx_sizes(int64_t rows, int64_t K, int fmt, int sf, size_t* code_bytes, size_t* scale_bytes) {
-    *code_bytes = (size_t)rows * (size_t)(fmt == LATMIX_MXFP4_E2M1 ? K / 2 : K);
-    if (sf == LATMIX_SF_LINEAR) *scale_bytes = (size_t)rows * (size_t)(K / 32);
+    *code_bytes = (size_t)rows * (size_t)(packs_two_codes(fmt) ? K / 2 : K);
+    if (fmt == LATMIX_NVFP4) *scale_bytes = nvfp4_block_scale_bytes(rows, K, sf) + kTensorScaleTrailerBytes;
+    else if (sf == LATMIX_SF_LINEAR) *scale_bytes = (size_t)rows * (size_t)(K / 32);
     else *scale_bytes = (size_t)((rows + 127) / 128) * (size_t)sf_k_tiles(K) * 512;
 }
 
 // Padding BLOCKS of the tiled scale layout (K/32 not a multiple of 8) are zeroed before the quantiser runs.  Padding ROWS
 // are not: whatever they hold scales accumulator rows (or columns) that lie outside the result and are never stored.
-static bool scales_have_block_padding(int64_t K, int sf) { return sf == LATMIX_SF_TCGEN05 && (K / 32) % 8 != 0; }
+static bool scales_have_block_padding(int64_t K, int sf, int fmt) {
+    return sf == LATMIX_SF_TCGEN05 && (fmt == LATMIX_NVFP4 ? (K / 16) % 16 != 0 : (K / 32) % 8 != 0);
+}
+// Zero the block-scale part of a scale buffer (never the NVFP4 trailer: the caller's tensor scale lives there).
+static cudaError_t zero_block_scales(void* scales, int64_t rows, int64_t K, int fmt, int sf, cudaStream_t st) {
+    size_t cb, sb;
+    mx_sizes(rows, K, fmt, sf, &cb, &sb);
+    if (fmt == LATMIX_NVFP4) sb -= kTensorScaleTrailerBytes;
+    return cudaMemsetAsync(scales, 0, sb, st);
+}
 
 }  // namespace latmix
 
@@ -69,6 +84,27 @@ size_t latmix_scale_offset(int64_t row, int64_t kblock, int64_t rows, int64_t K,
     if (!valid_sf(sf) || row < 0 || row >= rows || K <= 0 || K % 32 != 0 || kblock < 0 || kblock >= K / 32) return (size_t)-1;
     if (sf == LATMIX_SF_LINEAR) return (size_t)(row * (K / 32) + kblock);
     return sf_tcgen05_offset(row, kblock, sf_k_tiles(K));
+}
+
+size_t latmix_scale_offset_fmt(int64_t row, int64_t kblock, int64_t rows, int64_t K, latmix_format_t fmt, latmix_sf_layout_t sf) {
+    if (fmt != LATMIX_NVFP4) return valid_fmt(fmt) ? latmix_scale_offset(row, kblock, rows, K, sf) : (size_t)-1;
+    if (!valid_sf(sf) || row < 0 || row >= rows || K <= 0 || K % 64 != 0 || kblock < 0 || kblock >= K / 16) return (size_t)-1;
+    if (sf == LATMIX_SF_LINEAR) return (size_t)(row * (K / 16) + kblock);
+    return sf_tcgen05_offset(row, kblock, nvfp4_sf_k_tiles(K));
+}
+
+size_t latmix_tensor_scale_offset(int64_t rows, int64_t K, latmix_format_t fmt, latmix_sf_layout_t sf) {
+    if (fmt != LATMIX_NVFP4 || !valid_sf(sf) || rows < 0 || K < 0 || K % 64 != 0) return (size_t)-1;
+    return nvfp4_block_scale_bytes(rows, K, sf);
+}
+
+latmix_status_t latmix_workspace_set_tensor_scale(void* workspace, size_t workspace_bytes, float tensor_scale, void* cuda_stream) {
+    if (workspace == nullptr || workspace_bytes < kWorkspaceHeaderBytes) return LATMIX_ERR_WORKSPACE;
+    if (!aligned16(workspace) || !(tensor_scale > 0.0f) || !(tensor_scale < 3.0e38f)) return LATMIX_ERR_INVALID_ARG;
+    if (cudaMemcpyAsync(static_cast<uint8_t*>(workspace) + kHeaderTensorScaleOffset, &tensor_scale, sizeof(float), cudaMemcpyHostToDevice,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return LATMIX_ERR_CUDA;
+    return LATMIX_OK;
 }
 
 latmix_status_t latmix_workspace_bytes(latmix_op_t op, int64_t M, int64_t K, int64_t N, latmix_format_t fmt, size_t* bytes) {
@@ -174,12 +210,9 @@ latmix_status_t latmix_quantize_mx(const void* X, latmix_dtype_t x_dtype, const 
     if ((s = check_device()) != LATMIX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint32_t* status = static_cast<uint32_t*>(workspace);
-    if (scales_have_block_padding(K, sf)) {
-        size_t cb, sb;
-        mx_sizes(M, K, fmt, sf, &cb, &sb);
-        if (cudaMemsetAsync(scales, 0, sb, st) != cudaSuccess) return LATMIX_ERR_CUDA;
-    }
+    if (scales_have_block_padding(K, sf, fmt) && zero_block_scales(scales, M, K, fmt, sf, st) != cudaSuccess) return LATMIX_ERR_CUDA;
     cudaError_t e;
+    if (fmt == LATMIX_NVFP4 && (flags & LATMIX_FLAG_BLOCK_DIAG)) return LATMIX_ERR_UNSUPPORTED;
     if (A == nullptr || (flags & LATMIX_FLAG_BLOCK_DIAG)) {
         QuantArgs q{X, x_dtype == LATMIX_BF16, b, M, K, (int)fmt, (int)sf, static_cast<uint8_t*>(codes),
                     static_cast<uint8_t*>(scales), Y_dump, status, flags};
@@ -189,7 +222,13 @@ latmix_status_t latmix_quantize_mx(const void* X, latmix_dtype_t x_dtype, const 
                              Y_dump, status, flags};
         const bool tc = x_dtype == LATMIX_BF16 && !(flags & LATMIX_FLAG_FORCE_SIMT);
         const uint32_t variant = (flags >> 8) & 0xFu;       // tuning override: 1-3 = single-CTA kernel, 4 = small-batch kernel, 8 = CTA pairs
-        if (tc && (variant == 0 || variant == 4) && transform_quant_decode_tc_supported(t)) {
+        if (tc && fmt == LATMIX_NVFP4 && transform_quant_pair_tc_supported(t)) {
+            e = launch_transform_quant_pair_tc(t, st);      // the one tensor-core kernel whose epilogue knows blocks of 16
+        } else if (fmt == LATMIX_NVFP4) {
+            GemmQuantArgs g{X, x_dtype == LATMIX_BF16, K, 1, A, x_dtype == LATMIX_BF16, K, 1, b, M, K, K, (int)fmt, (int)sf,
+                            static_cast<uint8_t*>(codes), static_cast<uint8_t*>(scales), Y_dump, status, flags};
+            e = launch_gemm_quant_simt(g, st);
+        } else if (tc && (variant == 0 || variant == 4) && transform_quant_decode_tc_supported(t)) {
             e = launch_transform_quant_decode_tc(t, st);    // M <= 16: bound by reading A once
         } else if (tc && (variant == 0 || variant == 8) && transform_quant_pair_tc_supported(t)) {
             e = launch_transform_quant_pair_tc(t, st);
@@ -252,11 +291,7 @@ latmix_status_t latmix_fold_weights(const void* A_inv, const float* b, const voi
     if (N == 0 || K == 0) return LATMIX_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* base = static_cast<uint8_t*>(workspace);
-    if (scales_have_block_padding(K, sf)) {
-        size_t cb, sb;
-        mx_sizes(N, K, fmt, sf, &cb, &sb);
-        if (cudaMemsetAsync(Wq_scales, 0, sb, st) != cudaSuccess) return LATMIX_ERR_CUDA;
-    }
+    if (scales_have_block_padding(K, sf, fmt) && zero_block_scales(Wq_scales, N, K, fmt, sf, st) != cudaSuccess) return LATMIX_ERR_CUDA;
     return run_fold(static_cast<const float*>(A_inv), b, W, w_dtype, bias, K, N, fmt, sf, static_cast<uint8_t*>(Wq_codes),
                     static_cast<uint8_t*>(Wq_scales), c_out, Wfold_dump, static_cast<uint32_t*>(workspace),
                     reinterpret_cast<double*>(base + kWorkspaceHeaderBytes), workspace_bytes > need ? base + need : nullptr,
@@ -272,6 +307,7 @@ latmix_status_t latmix_fold_weights_two_sided(const float* A_in_inv, const float
         !valid_dtype(w_dtype) || !valid_sf(sf))
         return LATMIX_ERR_INVALID_ARG;
     if (A_in_inv == nullptr && A_out == nullptr) return LATMIX_ERR_INVALID_ARG;          // nothing to fold
+    if (fmt == LATMIX_NVFP4 && A_out != nullptr) return LATMIX_ERR_UNSUPPORTED;
     if ((A_in_inv == nullptr && b_in != nullptr) || (A_out == nullptr && v_out != nullptr)) return LATMIX_ERR_INVALID_ARG;
     if (!aligned16(A_in_inv) || !aligned16(b_in) || !aligned16(W) || !aligned16(bias) || !aligned16(A_out) || !aligned16(v_out) ||
         !aligned16(Wq_codes) || !aligned16(Wq_scales) || !aligned16(c_out) || !aligned16(Wfold_dump))
@@ -301,11 +337,7 @@ latmix_status_t latmix_fold_weights_two_sided(const float* A_in_inv, const float
     uint32_t* status = static_cast<uint32_t*>(workspace);
     uint8_t* codes = static_cast<uint8_t*>(Wq_codes);
     uint8_t* scales = static_cast<uint8_t*>(Wq_scales);
-    if (scales_have_block_padding(K, sf)) {
-        size_t cb, sb;
-        mx_sizes(N, K, fmt, sf, &cb, &sb);
-        if (cudaMemsetAsync(Wq_scales, 0, sb, st) != cudaSuccess) return LATMIX_ERR_CUDA;
-    }
+    if (scales_have_block_padding(K, sf, fmt) && zero_block_scales(Wq_scales, N, K, fmt, sf, st) != cudaSuccess) return LATMIX_ERR_CUDA;
     if (use_tc2) {
         float* T = nullptr;
         if (launch_fold_two_sided_tc(A_in_inv, W, A_out, K, N, (int)fmt, (int)sf, codes, scales, Wfold_dump, &T, status, flags,
@@ -350,6 +382,7 @@ latmix_status_t latmix_transformation_mse(const void* X, latmix_dtype_t x_dtype,
                                           void* cuda_stream) {
     if (X == nullptr || block_err == nullptr || mse == nullptr || !valid_fmt(fmt) || !valid_dtype(x_dtype)) return LATMIX_ERR_INVALID_ARG;
     if ((A == nullptr) != (A_inv == nullptr)) return LATMIX_ERR_INVALID_ARG;        // a transform comes with its inverse
+    if (fmt == LATMIX_NVFP4) return LATMIX_ERR_UNSUPPORTED;
     if (!aligned16(A_inv) || !aligned16(block_err) || (reinterpret_cast<uintptr_t>(mse) & 7u)) return LATMIX_ERR_INVALID_ARG;
     latmix_status_t s = shape_check(M, K, fmt);
     if (s != LATMIX_OK) return s;
@@ -411,13 +444,22 @@ static latmix_status_t run_mx_gemm(const void* a_codes, const void* a_scales, co
                  static_cast<const uint8_t*>(w_codes), static_cast<const uint8_t*>(w_scales), c, M, K, N,
                  // MXINT4 codes are the E4M3 bytes of the integers: the contraction is the MXFP8 one, products exact
                  fmt == LATMIX_MXINT4 ? (int)LATMIX_MXFP8_E4M3 : (int)fmt, out, ldo, static_cast<uint32_t*>(workspace), flags};
+    if (fmt == LATMIX_NVFP4) {
+        g.a_tensor_scale = nvfp4_tensor_scale_ptr(g.a_scales, M, K, LATMIX_SF_TCGEN05);
+        g.w_tensor_scale = nvfp4_tensor_scale_ptr(g.w_scales, N, K, LATMIX_SF_TCGEN05);
+        cudaError_t en = (!(flags & LATMIX_FLAG_FORCE_SIMT) && mx_gemm_wide_tc_supported(g)) ? launch_mx_gemm_wide_tc(g, st)
+                                                                                              : launch_mx_gemm_simt(g, st);
+        return en == cudaSuccess ? LATMIX_OK : LATMIX_ERR_CUDA;
+    }
     cudaError_t e;
-    // tuning override in flag bits 8-11: 0 = default choice (small-batch kernel for M <= 64, CTA pairs for M > 128, single
-    // CTA in between), 1-3 = single-CTA tile shapes, 4 = small-batch kernel, 8 = CTA pairs
+    // tuning override in flag bits 8-11: 0 = default choice (small-batch kernel for M <= 64, CTA pairs with 256 x 256 tiles for
+    // M > 128, single CTA in between), 1-3 = single-CTA tile shapes, 4 = small-batch kernel, 8 = CTA pairs with 256 x 192
+    // tiles, 9 = CTA pairs with 256 x 256 tiles
     const uint32_t variant = (flags >> 8) & 0xFu;
     const bool tc = !(flags & LATMIX_FLAG_FORCE_SIMT);
     if (tc && (variant == 0 || variant == 4) && mx_gemm_decode_tc_supported(g)) e = launch_mx_gemm_decode_tc(g, st);   // M <= 64
     else if (tc && (variant == 0 || variant == 4) && mxint8_gemm_decode_tc_supported(g)) e = launch_mxint8_gemm_decode_tc(g, st);   // MXINT8, M <= 16: no scratch
+    else if (tc && (variant == 0 || variant == 9) && mx_gemm_wide_tc_supported(g)) e = launch_mx_gemm_wide_tc(g, st);   // M > 128
     else if (tc && (variant == 0 || variant == 8) && mx_gemm_pair_tc_supported(g)) e = launch_mx_gemm_pair_tc(g, st);
     else if (tc && mx_gemm_tc_supported(g)) e = launch_mx_gemm_tc(g, st);
     else if (tc && mxint8_gemm_tc_supported(g) && scratch != nullptr && scratch_bytes >= mxint8_gemm_tc_scratch_bytes(M, K, N))
@@ -456,6 +498,15 @@ latmix_status_t latmix_linear(const void* X, latmix_dtype_t x_dtype, const void*
     if (Wq_codes == nullptr || Wq_scales == nullptr || out == nullptr || N < 0) return LATMIX_ERR_INVALID_ARG;
     if (!aligned16(Wq_codes) || !aligned16(Wq_scales) || !aligned16(c) || !aligned16(out)) return LATMIX_ERR_INVALID_ARG;
     if (ldo < N || ldo % 4 != 0) return LATMIX_ERR_SHAPE;
+    if (fmt == LATMIX_NVFP4) {
+        // the activations' tensor scale: from the workspace header (latmix_workspace_set_tensor_scale) to the trailer of
+        // the activation scale buffer, where the quantiser and the product look for it
+        if ((s = check_device()) != LATMIX_OK) return s;
+        if (M > 0 && K > 0 &&
+            cudaMemcpyAsync(a_scales + nvfp4_block_scale_bytes(M, K, LATMIX_SF_TCGEN05), base + kHeaderTensorScaleOffset, sizeof(float),
+                            cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+            return LATMIX_ERR_CUDA;
+    }
     s = latmix_quantize_mx(X, x_dtype, A, b, M, K, fmt, LATMIX_SF_TCGEN05, a_codes, a_scales, nullptr, workspace,
                            workspace_bytes, flags, cuda_stream);
     if (s != LATMIX_OK) return s;

@@ -10,6 +10,9 @@ namespace latmix {
 
 // The first 256 bytes of every workspace: word 0 is the device status (bitwise OR of 1 << latmix_status_t).
 constexpr size_t kWorkspaceHeaderBytes = 256;
+// Header layout: word 0 status, word 1 wait limit in cycles (0 = default), bytes 16-19 the NVFP4 tensor scale of the
+// activations that latmix_linear quantises (latmix_workspace_set_tensor_scale).
+constexpr size_t kHeaderTensorScaleOffset = 16;
 
 void count_launch(int n = 1);
 
@@ -60,6 +63,8 @@ struct MxGemmArgs {
     int fmt;
     float* out; int64_t ldo;
     uint32_t* status; uint32_t flags;
+    const float* a_tensor_scale = nullptr;      // NVFP4: the fp32 scale of each operand (device memory)
+    const float* w_tensor_scale = nullptr;
 };
 // CUDA-core block-scaled product: any shape; also the small-M (decode) path.
 cudaError_t launch_mx_gemm_simt(const MxGemmArgs& a, cudaStream_t st);
@@ -73,6 +78,10 @@ cudaError_t launch_mx_gemm_decode_tc(const MxGemmArgs& a, cudaStream_t st);
 // The same product on CTA pairs (cta_group::2, 256-row tiles): half the weight bytes per SM.
 bool mx_gemm_pair_tc_supported(const MxGemmArgs& a);
 cudaError_t launch_mx_gemm_pair_tc(const MxGemmArgs& a, cudaStream_t st);
+
+// CTA pairs with 256 x 256 tiles and two accumulators that overlap in tensor memory; also the NVFP4 product.
+bool mx_gemm_wide_tc_supported(const MxGemmArgs& a);
+cudaError_t launch_mx_gemm_wide_tc(const MxGemmArgs& a, cudaStream_t st);
 
 struct TransformQuantArgs {
     const void* X; const void* A;   // bf16, row-major M x K and K x K

@@ -11,7 +11,8 @@ namespace latmix {
 
 // FMT_INT4: integers k in [-7, 7], each stored as the E4M3 byte of k, so that the 8-bit block-scaled tensor-core kind
 // consumes the codes as they are (the products stay exact)
-enum : int { FMT_FP4 = 0, FMT_FP8 = 1, FMT_INT8 = 2, FMT_INT4 = 3 };
+// FMT_NVFP4: E2M1 elements packed like FMT_FP4, blocks of 16 with an E4M3 scale each, one fp32 scale per tensor
+enum : int { FMT_FP4 = 0, FMT_FP8 = 1, FMT_INT8 = 2, FMT_INT4 = 3, FMT_NVFP4 = 4 };
 
 // r_max of Eq. "q_mx": exponent of the top binade of the element format.
 template <int FMT> struct FormatTraits;
@@ -125,6 +126,38 @@ __host__ __device__ __forceinline__ size_t sf_tcgen05_offset(int64_t row, int64_
     return (size_t)((row >> 7) * k_tiles + (kb >> 2)) * 512 + (size_t)((row & 31) * 16 + ((row >> 5) & 3) * 4 + (kb & 3));
 }
 __host__ __device__ __forceinline__ int64_t sf_k_tiles(int64_t K) { return ((K / 32 + 7) / 8) * 2; }  // blocks padded to 8
+// NVFP4: a tile holds 128 rows x 4 blocks of 16 elements; blocks padded to 16, i.e. k-tiles to a multiple of 4 (one 128-byte slab)
+__host__ __device__ __forceinline__ int64_t nvfp4_sf_k_tiles(int64_t K) { return ((K / 16 + 15) / 16) * 4; }
+
+// NVFP4 scale buffers end with a 16-byte trailer whose first four bytes hold the tensor's fp32 scale; this is the
+// trailer's offset, i.e. the bytes the block scales take (linear: rows x K/16 bytes rounded up to 16; tiled: whole tiles).
+__host__ __device__ __forceinline__ size_t nvfp4_block_scale_bytes(int64_t rows, int64_t K, int sf_layout) {
+    return sf_layout == 0 ? (size_t)((rows * (K / 16) + 15) / 16 * 16) : (size_t)((rows + 127) / 128) * (size_t)nvfp4_sf_k_tiles(K) * 512;
+}
+__host__ __device__ __forceinline__ const float* nvfp4_tensor_scale_ptr(const uint8_t* scales, int64_t rows, int64_t K, int sf_layout) {
+    return reinterpret_cast<const float*>(scales + nvfp4_block_scale_bytes(rows, K, sf_layout));
+}
+
+// One NVFP4 block: 16 fp32 values -> the block's E4M3 scale code and eight bytes of E2M1 codes, for tensor scale g.
+// fp32 arithmetic, one IEEE operation per step, in this order (no fused multiply-add, no reciprocal approximation):
+//   t = (amax / 6) / g;  d = E4M3(t), round to nearest even, saturating;  s = d * g;  r = 1 / s (0 if s == 0);
+//   code_j = E2M1(v_j * r), round to nearest even, saturating, sign kept.
+__device__ __forceinline__ uint32_t nvfp4_quantize_block(const float* v, float g, uint2& packed) {
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+    const float t = __fdiv_rn(__fdiv_rn(amax, 6.0f), g);
+    const uint32_t d_code = (uint32_t)__nv_cvt_float_to_fp8(t, __NV_SATFINITE, __NV_E4M3) & 0xFFu;
+    const uint32_t e = (d_code >> 3) & 15u, m = d_code & 7u;
+    const float d = e == 0 ? (float)m * 0.001953125f : __uint_as_float(((e + 120u) << 23) | (m << 20));
+    const float s = __fmul_rn(d, g);
+    const float r = s > 0.f ? __fdiv_rn(1.0f, s) : 0.f;
+    float w[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) w[i] = __fmul_rn(v[i], r);
+    packed = make_uint2(pack8_fp4(w), pack8_fp4(w + 8));
+    return d_code;
+}
 
 // 2^(E-6) for scale byte E + 127, exact (byte 0: 2^-133, a subnormal)
 __device__ __forceinline__ float int8_mult(uint32_t scale_byte) { return scale_to_float(scale_byte) * 0.015625f; }

@@ -62,13 +62,58 @@ __global__ void __launch_bounds__(kProbeThreads, 1) tensor_pipe_probe_kernel(lon
     if (warp_idx == 0) tmem_dealloc(tmem_base, 512);
 }
 
+// The same probe on a CTA pair: one 256 x 256 x 64 kind::mxf4 MMA per step (cta_group::2), each CTA holding its 128 rows of
+// A and half of the rows of B; the leader issues, both tensor cores work.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kProbeThreads, 1) tensor_pipe_probe_pair_kernel(long long mma_per_pair, int commit_every, uint32_t* status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    constexpr int kA = 128 * 128, kBhalf = 128 * 128;
+    const uint32_t sf_base = smem_base + kA + kBhalf, bar = sf_base + kProbeSf, tmem_slot = bar + 8, bar2 = bar + 16;
+    const int warp_idx = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool leader = cluster_ctarank() == 0;
+    for (int i = threadIdx.x; i < (kA + kBhalf) / 4; i += kProbeThreads)
+        reinterpret_cast<uint32_t*>(smem_gen)[i] = 0x38383838u | ((uint32_t)(i * 2654435761u) & 0x07070707u);
+    for (int i = threadIdx.x; i < kProbeSf / 4; i += kProbeThreads)
+        reinterpret_cast<uint32_t*>(smem_gen + kA + kBhalf)[i] = 0x7F7F7F7Fu;
+    if (threadIdx.x == 0) { mbar_init(bar, 1); mbar_init(bar2, 1); fence_mbar_init(); }
+    fence_proxy_async_smem();
+    if (warp_idx == 0) { tmem_alloc_pair(tmem_slot, 512); tmem_relinquish_pair(); }
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
+    if (leader && warp_idx == 1 && lane == 0) {
+        const uint32_t sfa_t = tmem_base + 256, sfb_t = tmem_base + 260;
+        tc_cp_scale_pair_lean(sfa_t, desc_lo(sf_base));
+        tc_cp_scale_pair_lean(sfb_t, desc_lo(sf_base + 512));
+        tc_cp_scale_pair_lean(sfb_t + 4, desc_lo(sf_base + 1024));
+        const uint32_t a_lo = desc_lo(smem_base), b_lo = desc_lo(smem_base + kA);
+        constexpr uint32_t kIdMx = make_idesc_block_scaled(256, 256, 1u);
+        for (long long i = 0; i < mma_per_pair; i += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                mma_mxf4_pair_lean(tmem_base, a_lo + 2 * j, b_lo + 2 * j, (j & 1) ? (kIdMx | (2u << 4) | (2u << 29)) : kIdMx, sfa_t, sfb_t, (i | j) != 0);
+            // a commit every so many MMAs, as a pipelined kernel issues them to release its stages (nobody waits on this one)
+            if (commit_every > 0 && (i + 4) % commit_every == 0) tc_commit_pair(bar2, 1);
+        }
+        tc_commit_pair(bar, 1);
+        mbar_wait(bar, 0, status);
+    }
+    tc_fence_before();
+    cluster_sync_all();                 // the peer's shared and tensor memory stay until the leader's MMAs are done
+    if (warp_idx == 0) tmem_dealloc_pair(tmem_base, 512);
+}
+
 }  // namespace latmix
 
 using namespace latmix;
 
-extern "C" latmix_status_t latmix_tensor_pipe_probe(int kind, int64_t mma_per_cta, double* flops, void* workspace,
+extern "C" latmix_status_t latmix_tensor_pipe_probe(int kind_and_interval, int64_t mma_per_cta, double* flops, void* workspace,
                                                     size_t workspace_bytes, void* cuda_stream) {
-    if (kind < 0 || kind > 3 || mma_per_cta < 4 || mma_per_cta > (1ll << 22) || flops == nullptr) return LATMIX_ERR_INVALID_ARG;
+    const int kind = kind_and_interval & 0xFF, commit_every = (kind_and_interval >> 8) & 0xFFFF;
+    if (commit_every != 0 && (kind != 4 || commit_every % 4 != 0)) return LATMIX_ERR_INVALID_ARG;
+    if (kind < 0 || kind > 4 || mma_per_cta < 4 || mma_per_cta > (1ll << 22) || flops == nullptr) return LATMIX_ERR_INVALID_ARG;
     if (workspace == nullptr || workspace_bytes < kWorkspaceHeaderBytes || (reinterpret_cast<uintptr_t>(workspace) & 15u))
         return LATMIX_ERR_WORKSPACE;
     int dev = 0, major = 0, sms = 0;
@@ -85,7 +130,12 @@ extern "C" latmix_status_t latmix_tensor_pipe_probe(int kind, int64_t mma_per_ct
         e = cudaFuncSetAttribute(tensor_pipe_probe_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kProbeSmem); \
         if (e == cudaSuccess) tensor_pipe_probe_kernel<KIND><<<sms, kProbeThreads, kProbeSmem, st>>>(n, status);        \
     } while (0)
-    if (kind == 0) LATMIX_PROBE(0); else if (kind == 1) LATMIX_PROBE(1); else if (kind == 2) LATMIX_PROBE(2); else LATMIX_PROBE(3);
+    if (kind == 0) LATMIX_PROBE(0); else if (kind == 1) LATMIX_PROBE(1); else if (kind == 2) LATMIX_PROBE(2); else if (kind == 3) LATMIX_PROBE(3);
+    else {
+        e = cudaFuncSetAttribute(tensor_pipe_probe_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kProbeSmem);
+        sms = 2 * resident_cta_pairs((const void*)tensor_pipe_probe_pair_kernel, kProbeThreads, kProbeSmem);
+        if (e == cudaSuccess) tensor_pipe_probe_pair_kernel<<<sms, kProbeThreads, kProbeSmem, st>>>(n, commit_every, status);
+    }
 #undef LATMIX_PROBE
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return LATMIX_ERR_CUDA;
     count_launch();

@@ -15,7 +15,27 @@ namespace latmix {
 template <int FMT>
 __device__ __forceinline__ void quantize_block_by_4_lanes(float (&v)[8], bool active, int64_t row, int64_t k0,
                                                           int64_t K, uint8_t* codes, uint8_t* scales, int sf_layout,
-                                                          uint32_t* status, uint32_t flags) {
+                                                          uint32_t* status, uint32_t flags, int64_t rows_total) {
+    if (FMT == FMT_NVFP4) {
+        // a block of 16 = two neighbouring lanes: the even lane fetches its neighbour's eight values and quantises the block
+        float w[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { w[i] = v[i]; w[8 + i] = __shfl_down_sync(0xffffffffu, v[i], 1); }
+        if ((flags & LATMIX_FLAG_CHECK_FINITE) && active) {
+            bool bad = false;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) bad |= !isfinite(v[i]);
+            if (bad) atomicOr(status, 1u << LATMIX_ERR_NONFINITE);
+        }
+        if (!active || (k0 & 15) != 0) return;
+        const float g = *nvfp4_tensor_scale_ptr(scales, rows_total, K, sf_layout);
+        uint2 packed;
+        const uint32_t d_code = nvfp4_quantize_block(w, g, packed);
+        *reinterpret_cast<uint2*>(codes + row * (K >> 1) + (k0 >> 1)) = packed;
+        const int64_t kb = k0 >> 4;
+        scales[sf_layout == LATMIX_SF_LINEAR ? (size_t)(row * (K >> 4) + kb) : sf_tcgen05_offset(row, kb, nvfp4_sf_k_tiles(K))] = (uint8_t)d_code;
+        return;
+    }
     float amax = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
@@ -27,12 +47,12 @@ __device__ __forceinline__ void quantize_block_by_4_lanes(float (&v)[8], bool ac
         for (int i = 0; i < 8; ++i) bad |= !isfinite(v[i]);
         if (bad) atomicOr(status, 1u << LATMIX_ERR_NONFINITE);
     }
-    const uint32_t sb = scale_byte_from_amax(amax, FormatTraits<FMT>::kRMax);
+    const uint32_t sb = scale_byte_from_amax(amax, FormatTraits<FMT == FMT_NVFP4 ? FMT_FP4 : FMT>::kRMax);
     const float2 f = inv_scale_factors(sb);
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = (v[i] * f.x) * f.y;
     if (!active) return;
-    if (FMT == FMT_FP4) {
+    if (FMT == FMT_FP4 || FMT == FMT_NVFP4) {
         *reinterpret_cast<uint32_t*>(codes + row * (K >> 1) + (k0 >> 1)) = pack8_fp4(v);
     } else {
         *reinterpret_cast<uint2*>(codes + row * K + k0) = pack8_bytes<FMT>(v);
@@ -170,8 +190,56 @@ __global__ void __launch_bounds__(256, 4) quantize_rows_kernel(const TIn* __rest
     }
 }
 
+// NVFP4 (blocks of 16, E4M3 block scale, tensor scale from the scale buffer's trailer): a thread = one block.
+template <typename TIn>
+__global__ void __launch_bounds__(256) quantize_rows_nvfp4_kernel(const TIn* __restrict__ X, const float* __restrict__ b, int64_t M,
+                                                                  int64_t K, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                                                                  int sf_layout, float* __restrict__ Y_dump, uint32_t* status,
+                                                                  uint32_t flags) {
+    const float g = *nvfp4_tensor_scale_ptr(scales, M, K, sf_layout);
+    const int64_t nb = K >> 4, total = M * nb, kt = nvfp4_sf_k_tiles(K);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / nb, kb = i - row * nb, k0 = kb << 4;
+        float v[16];
+        load8(X + row * K + k0, *reinterpret_cast<float(*)[8]>(v));
+        load8(X + row * K + k0 + 8, *reinterpret_cast<float(*)[8]>(v + 8));
+        if (b != nullptr) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] += b[k0 + j];
+        }
+        if (Y_dump != nullptr) {
+            float4* d = reinterpret_cast<float4*>(Y_dump + row * K + k0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) d[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        }
+        if (flags & LATMIX_FLAG_CHECK_FINITE) {
+            bool bad = false;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) bad |= !isfinite(v[j]);
+            if (bad) atomicOr(status, 1u << LATMIX_ERR_NONFINITE);
+        }
+        uint2 packed;
+        const uint32_t d_code = nvfp4_quantize_block(v, g, packed);
+        *reinterpret_cast<uint2*>(codes + row * (K >> 1) + (k0 >> 1)) = packed;
+        scales[sf_layout == LATMIX_SF_LINEAR ? (size_t)(row * nb + kb) : sf_tcgen05_offset(row, kb, kt)] = (uint8_t)d_code;
+    }
+}
+
 cudaError_t launch_quantize_rows(const QuantArgs& a, cudaStream_t st) {
     if (a.M == 0 || a.K == 0) return cudaSuccess;
+    if (a.fmt == FMT_NVFP4) {
+        const int64_t total = a.M * (a.K >> 4);
+        int64_t blocks = (total + 255) / 256;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        if (a.x_is_bf16)
+            quantize_rows_nvfp4_kernel<<<(unsigned)blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(a.X), a.b, a.M, a.K, a.codes, a.scales,
+                                                                        a.sf_layout, a.Y_dump, a.status, a.flags);
+        else
+            quantize_rows_nvfp4_kernel<<<(unsigned)blocks, 256, 0, st>>>(static_cast<const float*>(a.X), a.b, a.M, a.K, a.codes, a.scales,
+                                                                        a.sf_layout, a.Y_dump, a.status, a.flags);
+        count_launch();
+        return cudaGetLastError();
+    }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -376,7 +444,7 @@ __global__ void __launch_bounds__(256) gemm_quant_simt_kernel(const TP* __restri
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = 0.f;
         }
-        quantize_block_by_4_lanes<FMT>(v, active, gr, gk, C, codes, scales, sf_layout, status, flags);
+        quantize_block_by_4_lanes<FMT>(v, active, gr, gk, C, codes, scales, sf_layout, status, flags, R);
     }
 }
 
@@ -408,6 +476,7 @@ cudaError_t launch_gemm_quant_simt(const GemmQuantArgs& a, cudaStream_t st) {
     if (a.fmt == FMT_FP4) launch_gq_fmt<FMT_FP4>(a, st);
     else if (a.fmt == FMT_FP8) launch_gq_fmt<FMT_FP8>(a, st);
     else if (a.fmt == FMT_INT4) launch_gq_fmt<FMT_INT4>(a, st);
+    else if (a.fmt == FMT_NVFP4) launch_gq_fmt<FMT_NVFP4>(a, st);
     else launch_gq_fmt<FMT_INT8>(a, st);
     count_launch();
     return cudaGetLastError();
@@ -554,8 +623,44 @@ __global__ void __launch_bounds__(256) mx_gemm_simt_kernel(const uint8_t* __rest
     }
 }
 
+// NVFP4 on the CUDA cores: one warp per output column, a lane per block of 16; out = (ga gw) sum + c.
+__global__ void __launch_bounds__(256) nvfp4_gemm_simt_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ a_scales,
+                                                              const uint8_t* __restrict__ w_codes, const uint8_t* __restrict__ w_scales,
+                                                              const float* __restrict__ ga, const float* __restrict__ gw,
+                                                              const float* __restrict__ c, int64_t M, int64_t K, int64_t N,
+                                                              float* __restrict__ out, int64_t ldo) {
+    const int lane = threadIdx.x & 31;
+    const int64_t n = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (n >= N) return;
+    const int64_t nkb = K >> 4, kt = nvfp4_sf_k_tiles(K), row_bytes = K >> 1;
+    const float g = *ga * *gw;
+    for (int64_t m = blockIdx.y; m < M; m += gridDim.y) {
+        float acc = 0.f;
+        for (int64_t kb = lane; kb < nkb; kb += 32) {
+            const uint2 wq = *reinterpret_cast<const uint2*>(w_codes + n * row_bytes + kb * 8);
+            const uint2 aq = *reinterpret_cast<const uint2*>(a_codes + m * row_bytes + kb * 8);
+            const uint32_t ww[2] = {wq.x, wq.y}, aw[2] = {aq.x, aq.y};
+            float s = 0.f;
+#pragma unroll
+            for (int t = 0; t < 16; ++t)
+                s = fmaf(decode_element<FMT_FP4>((aw[t >> 3] >> (4 * (t & 7))) & 0xFu), decode_element<FMT_FP4>((ww[t >> 3] >> (4 * (t & 7))) & 0xFu), s);
+            acc = fmaf(s, decode_element<FMT_FP8>(a_scales[sf_tcgen05_offset(m, kb, kt)]) * decode_element<FMT_FP8>(w_scales[sf_tcgen05_offset(n, kb, kt)]), acc);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) out[m * ldo + n] = fmaf(acc, g, c != nullptr ? c[n] : 0.f);
+    }
+}
+
 cudaError_t launch_mx_gemm_simt(const MxGemmArgs& a, cudaStream_t st) {
     if (a.M == 0 || a.N == 0) return cudaSuccess;
+    if (a.fmt == FMT_NVFP4) {
+        dim3 grid((unsigned)((a.N + 7) / 8), (unsigned)(a.M < 1024 ? a.M : 1024));
+        nvfp4_gemm_simt_kernel<<<grid, 256, 0, st>>>(a.a_codes, a.a_scales, a.w_codes, a.w_scales, a.a_tensor_scale, a.w_tensor_scale, a.c,
+                                                     a.M, a.K, a.N, a.out, a.ldo);
+        count_launch();
+        return cudaGetLastError();
+    }
     int64_t gy = (a.M + SG_ROWS - 1) / SG_ROWS;
     if (gy > 512) gy = 512;
     dim3 grid((unsigned)((a.N + 7) / 8), (unsigned)gy), block(256);

@@ -53,6 +53,7 @@ extern "C" latmix_status_t latmix_linear_static(const void* X, latmix_dtype_t x_
                                                 const void* Wq_codes, const void* Wq_scales, const float* c, int64_t M,
                                                 int64_t K, int64_t N, latmix_format_t fmt, float* out, int64_t ldo,
                                                 uint32_t flags, latmix_status_t* device_status, void* cuda_stream) {
+    if (fmt == LATMIX_NVFP4) return LATMIX_ERR_UNSUPPORTED;     // its tensor scale would need the header this call clears
     // what latmix_linear cannot do without: the header, the activation codes and their scales
     size_t code_bytes = 0, scale_bytes = 0;
     latmix_status_t s = latmix_mx_sizes(M, K, fmt, LATMIX_SF_TCGEN05, &code_bytes, &scale_bytes);

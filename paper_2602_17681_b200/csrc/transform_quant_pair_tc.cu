@@ -230,7 +230,9 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
     } else {
         // ------------------------------------------------------------------ quantising epilogue (warps 2..5, both CTAs)
         const int q = warp_idx & 3;                                  // tensor-memory lane quarter this warp may read
-        constexpr int kRMax = FormatTraits<FMT>::kRMax;
+        constexpr int kRMax = FormatTraits<FMT == FMT_NVFP4 ? FMT_FP4 : FMT>::kRMax;
+        float nv_g = 1.0f;                                           // NVFP4: the tensor scale, from the scale buffer's trailer
+        if (FMT == FMT_NVFP4 && p.codes != nullptr) nv_g = *nvfp4_tensor_scale_ptr(p.scales, p.M, p.K, p.sf_layout);
         uint32_t item_count = 0;
         bool ok = true;
         for (int item = pair; item < p.num_items && ok; item += num_pairs, ++item_count) {
@@ -271,12 +273,25 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
                 }
                 if ((p.flags & LATMIX_FLAG_CHECK_FINITE) && blk_ok && !isfinite(amax)) atomicOr(p.status, 1u << LATMIX_ERR_NONFINITE);
                 if (p.codes == nullptr) continue;                // product only: the dump above is the result
+                if (FMT == FMT_NVFP4) {
+                    // two blocks of 16 per thread; their scale bytes are neighbours in both layouts
+                    uint2 w0, w1;
+                    const uint32_t s0 = nvfp4_quantize_block(v, nv_g, w0), s1 = nvfp4_quantize_block(v + 16, nv_g, w1);
+                    if (blk_ok) {
+                        *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (col0 >> 1)) = make_uint4(w0.x, w0.y, w1.x, w1.y);
+                        const int64_t kblk = col0 >> 4;
+                        const size_t off = p.sf_layout == LATMIX_SF_LINEAR ? (size_t)(row * (p.K >> 4) + kblk)
+                                                                           : sf_tcgen05_offset(row, kblk, p.sf_kt_total);
+                        *reinterpret_cast<uint16_t*>(p.scales + off) = (uint16_t)(s0 | (s1 << 8));
+                    }
+                    continue;
+                }
                 const uint32_t sb = scale_byte_from_amax(amax, kRMax);
                 const float2 f = inv_scale_factors(sb);
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = (v[i] * f.x) * f.y;
                 if (blk_ok) {
-                    if (FMT == FMT_FP4) {
+                    if (FMT == FMT_FP4 || FMT == FMT_NVFP4) {
                         uint4 w = make_uint4(pack8_fp4(v), pack8_fp4(v + 8), pack8_fp4(v + 16), pack8_fp4(v + 24));
                         *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (col0 >> 1)) = w;
                     } else {
@@ -333,12 +348,13 @@ cudaError_t launch_transform_quant_pair_tc(const TransformQuantArgs& a, cudaStre
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
     p.m_tiles = (int)((a.M + 255) / 256);
     p.n_tiles = (int)((a.K + BLOCK_N - 1) / BLOCK_N);
-    p.sf_layout = a.sf_layout; p.sf_kt_total = (int)sf_k_tiles(a.K);
+    p.sf_layout = a.sf_layout; p.sf_kt_total = (int)(a.fmt == FMT_NVFP4 ? nvfp4_sf_k_tiles(a.K) : sf_k_tiles(a.K));
     p.status = a.status; p.flags = a.flags;
     p.term_rows = 0; p.num_terms = 0; p.wrap = 1;
     const void* kern = a.fmt == FMT_FP4 ? (const void*)transform_quant_pair_tc_kernel<FMT_FP4, false>
                      : a.fmt == FMT_FP8 ? (const void*)transform_quant_pair_tc_kernel<FMT_FP8, false>
                      : a.fmt == FMT_INT4 ? (const void*)transform_quant_pair_tc_kernel<FMT_INT4, false>
+                     : a.fmt == FMT_NVFP4 ? (const void*)transform_quant_pair_tc_kernel<FMT_NVFP4, false>
                                         : (const void*)transform_quant_pair_tc_kernel<FMT_INT8, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -400,11 +416,12 @@ static cudaError_t launch_fold_product(const FoldProductArgs& a, cudaStream_t st
     p.num_kb = (int)((a.red_len + SLAB_K - 1) / SLAB_K);
     p.m_tiles = (int)((a.R + 255) / 256);
     p.n_tiles = (int)((a.C + BLOCK_N - 1) / BLOCK_N);
-    p.sf_layout = a.sf_layout; p.sf_kt_total = (int)sf_k_tiles(a.C);
+    p.sf_layout = a.sf_layout; p.sf_kt_total = (int)(a.fmt == FMT_NVFP4 ? nvfp4_sf_k_tiles(a.C) : sf_k_tiles(a.C));
     p.status = a.status; p.flags = a.flags;
     const void* kern = a.fmt == FMT_FP4 ? (const void*)transform_quant_pair_tc_kernel<FMT_FP4, true>
                      : a.fmt == FMT_FP8 ? (const void*)transform_quant_pair_tc_kernel<FMT_FP8, true>
                      : a.fmt == FMT_INT4 ? (const void*)transform_quant_pair_tc_kernel<FMT_INT4, true>
+                     : a.fmt == FMT_NVFP4 ? (const void*)transform_quant_pair_tc_kernel<FMT_NVFP4, true>
                                         : (const void*)transform_quant_pair_tc_kernel<FMT_INT8, true>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;

@@ -39,6 +39,18 @@ def test_sizes_and_scale_offsets(B):
     # padding: 130 rows -> 2 row tiles; 96 elements = 3 blocks -> 8 blocks = 2 k-tiles
     assert B.mx_sizes(130, 96, B.MXINT8, B.SF_TCGEN05) == (130 * 96, 2 * 2 * 512)
     assert B.mx_sizes(130, 96, B.MXINT4, B.SF_TCGEN05) == (130 * 96, 2 * 2 * 512)     # one E4M3 byte per element
+    # NVFP4: blocks of 16 (tiles of 128 rows x 4 blocks, blocks padded to 16), plus the 16-byte tensor-scale trailer
+    assert B.mx_sizes(4096, 4096, B.NVFP4, B.SF_TCGEN05) == (4096 * 2048, 32 * 64 * 512 + 16)
+    assert B.mx_sizes(130, 192, B.NVFP4, B.SF_TCGEN05) == (130 * 96, 2 * 4 * 512 + 16)
+    assert B.mx_sizes(3, 64, B.NVFP4, B.SF_LINEAR) == (3 * 32, 16 + 16)
+    assert B.tensor_scale_offset(130, 192, B.NVFP4, B.SF_TCGEN05) == 2 * 4 * 512
+    assert B.tensor_scale_offset(130, 192, B.MXFP4, B.SF_TCGEN05) == ctypes.c_size_t(-1).value
+    assert B.scale_offset_fmt(129, 5, 130, 192, B.NVFP4, B.SF_TCGEN05) == (1 * 4 + 1) * 512 + 1 * 16 + 0 * 4 + 1
+    assert B.scale_offset_fmt(129, 5, 130, 192, B.NVFP4, B.SF_LINEAR) == 129 * 12 + 5
+    assert B.scale_offset_fmt(0, 12, 130, 192, B.NVFP4, B.SF_LINEAR) == ctypes.c_size_t(-1).value
+    assert B.scale_offset_fmt(7, 3, 130, 192, B.MXFP8, B.SF_TCGEN05) == B.scale_offset(7, 3, 130, 192, B.SF_TCGEN05)
+    with pytest.raises(B.LatmixError):
+        B.mx_sizes(4, 96, B.NVFP4)
     rows, K = 300, 1088
     seen = set()
     cb, sb = B.mx_sizes(rows, K, B.MXFP8, B.SF_TCGEN05)

@@ -397,7 +397,8 @@ def test_fold_weights_two_sided_argument_rules(B):
 
 
 # ------------------------------------------------------------------ S3: block-scaled GEMM
-@pytest.mark.parametrize("fmt,variant", [(0, 0), (0, 1), (0, 2), (0, 3), (1, 0), (1, 1), (1, 3), (0, 8), (1, 8), (3, 0), (3, 1)])
+@pytest.mark.parametrize("fmt,variant", [(0, 0), (0, 1), (0, 2), (0, 3), (1, 0), (1, 1), (1, 3), (0, 8), (1, 8), (3, 0), (3, 1),
+                                         (0, 9), (1, 9), (3, 9)])
 def test_mx_gemm_tensor_core(B, fmt, variant):
     M, K, N = 300, 2048, 712                   # ragged M and N tails for every tile width, 8 or 16 k-slabs
     ac, asc = H.random_mx(M, K, fmt, 11)
@@ -416,11 +417,14 @@ def test_mx_gemm_tensor_core(B, fmt, variant):
 
 
 @pytest.mark.parametrize("fmt", [0, 1])
-@pytest.mark.parametrize("M,K,N", [(520, 1536, 392), (129, 256, 64), (1024, 512, 1024), (4096, 256, 3840), (2304, 768, 1000)])
-def test_mx_gemm_cta_pairs(B, fmt, M, K, N):
-    """The CTA-pair kernel: odd slab counts, a second CTA with a single valid row, fewer weight rows than one tile, whole
-    tiles, and several tiles per CTA pair (320 and 54 tiles on at most 74 pairs) so that both tile streams and both
-    accumulators are in use at once."""
+@pytest.mark.parametrize("kernel", [8, 9])
+@pytest.mark.parametrize("M,K,N", [(520, 1536, 392), (129, 256, 64), (1024, 512, 1024), (4096, 256, 3840), (2304, 768, 1000),
+                                   (2560, 2048, 8192)])
+def test_mx_gemm_cta_pairs(B, fmt, kernel, M, K, N):
+    """The CTA-pair kernels (8: 256 x 192 tiles, 9: 256 x 256 tiles as two halves in three rotating accumulators, the second
+    half catching up on the first at tile boundaries): odd slab counts, a second CTA with a single valid row, fewer weight rows than one tile, whole
+    tiles, and several tiles per CTA pair (up to 320 tiles on at most 74 pairs) so that both tile streams, both
+    accumulators and every wrap of the rings are in use at once."""
     ac, asc = H.random_mx(M, K, fmt, 31)
     wc, wsc = H.random_mx(N, K, fmt, 32)
     c = (torch.randn(N) * 0.1).float()
@@ -428,10 +432,13 @@ def test_mx_gemm_cta_pairs(B, fmt, M, K, N):
     dw, dsw = H.mx_to_device(B, wc, wsc, fmt)
     ws = B.new_workspace(B.OP_MX_GEMM, M, K, N, fmt)
     out = torch.full((M, N), float("nan"), device="cuda")
-    B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, out=out, ws=ws, flags=8 << 8)
+    B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, out=out, ws=ws, flags=kernel << 8)
     assert B.device_status(ws) == B.OK
     ref = orc.mx_matmul(ac, asc, wc, wsc, c.numpy(), H.FMT_NAME[fmt])
-    H.assert_gemm_parity(out.cpu().numpy(), ref, ac, asc, wc, wsc, H.FMT_NAME[fmt], K, c.numpy(), tag="pairs")
+    H.assert_gemm_parity(out.cpu().numpy(), ref, ac, asc, wc, wsc, H.FMT_NAME[fmt], K, c.numpy(), tag=f"pairs kernel {kernel}")
+    # same sums in the same order per output element as the single-CTA kernel: identical bits
+    out1 = B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, ws=ws, flags=1 << 8)
+    assert torch.equal(out, out1)
 
 
 def test_mx_gemm_padded_leading_dimension_and_no_bias(B):
