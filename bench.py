@@ -463,11 +463,22 @@ def run_fold(args, cfg, local_rank):
     if args.op == "mse":
         M = cfg.M
         X = synth.make_activations(M, K, cfg.seed, cfg.act, cfg.outlier_frac, cfg.outlier_scale, cfg.x_dtype, dev)
-        A = synth.make_transform(K, cfg.seed, cfg.x_dtype, cfg.b_std, dev)[0]
+        mse_flags = 0
+        if args.mse_transform == "identity":
+            A = A_inv = b_t = None
+        elif args.mse_transform == "hadamard":
+            A, b_t, A_inv = synth.make_block_transform(K, cfg.seed, "hadamard", a_dtype=cfg.x_dtype, device=dev)
+            mse_flags = B.FLAG_BLOCK_DIAG
+        else:
+            A, b_t, A_inv = synth.make_transform(K, cfg.seed, cfg.x_dtype, cfg.b_std, dev)
         ws = B.new_workspace(B.OP_TRANSFORMATION_MSE, M, K, 0, fmt, dev)
-        call = lambda: B.transformation_mse(X, A, layer["b"], layer["A_inv"], fmt, ws=ws)
-        flops = 2.0 * M * K * K * 2                              # the transform and the back-mapping product
-        issued = 2.0 * M * K * K * (1 + 9)                       # back-mapping: both operands as three bf16 terms
+        mse_out = {}
+
+        def call():
+            mse_out["mse"], mse_out["blk"] = B.transformation_mse(X, A, b_t, A_inv, fmt, ws=ws, flags=mse_flags, block=args.block)
+        n_prod = {"identity": 0, "hadamard": 1, "full": 2}[args.mse_transform]
+        flops = 2.0 * M * K * K * n_prod                         # the transform and the back-mapping product
+        issued = 2.0 * M * K * K * ({"identity": 0, "hadamard": 9, "full": 1 + 9}[args.mse_transform])   # back-mapping: three bf16 terms per operand
     elif two:
         A_out, v_out, _ = synth.make_transform(N, cfg.seed + 1, "f32", device=dev)
         ws = B.new_workspace(B.OP_FOLD_TWO_SIDED, 0, K, N, fmt, dev)
@@ -505,8 +516,10 @@ def run_fold(args, cfg, local_rank):
         "metric": "transformation MSE diagnostic time" if args.op == "mse" else "offline fold + weight quantisation time", "value": ms, "unit": "ms", "n_gpus": 1, "steps": steps,
         "warmup": warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 x 3-term bf16 -> f32", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "op": args.op, "weights": args.weights, "algorithmic_gflop": flops / 1e9,
-                   "issued_bf16_gflop": issued / 1e9, "l2": "operands larger than L2"},
+        "config": dict({"workload": workload_name(cfg), "op": args.op, "weights": args.weights, "algorithmic_gflop": flops / 1e9,
+                        "issued_bf16_gflop": issued / 1e9, "l2": "operands larger than L2"},
+                       **({"block": args.block, "transform": args.mse_transform, "transformation_mse": float(mse_out["mse"]),
+                           "block_err_min_max": [float(mse_out["blk"].min()), float(mse_out["blk"].max())]} if args.op == "mse" else {})),
         "clocks": clocks, "gpu_launches": int(B.launch_count() - n0),
         "roofline": {"bound": "tensor", "achieved": issued / (ms * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                      "frac": issued / (ms * 1e-3) / 1e12 / peak, "traffic": None,

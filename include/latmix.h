@@ -225,6 +225,18 @@ latmix_status_t latmix_transformation_mse(const void* X, latmix_dtype_t x_dtype,
                                           void* cuda_stream);
 
 /*
+ * The same diagnostic for another MX block size B (8, 16, 32, 64 or 128; K a multiple of B): the sweep over block sizes of
+ * the numerical analysis in Sec. 3.1 (MSE against block size, block-wise error against block index).  y is computed as
+ * above; its quantisation Q_B follows Eq. "q_mx" with blocks of B elements; block_err has K/B entries, each the mean over
+ * the rows and the B coordinates of that block.  B = 32 is latmix_transformation_mse.  The block-scaled product of the layer
+ * always works with B = 32: other sizes exist for this diagnostic only.
+ */
+latmix_status_t latmix_transformation_mse_block(const void* X, latmix_dtype_t x_dtype, const void* A, const float* b,
+                                                const float* A_inv, int64_t M, int64_t K, latmix_format_t fmt, int block,
+                                                double* block_err, double* mse, void* workspace, size_t workspace_bytes,
+                                                uint32_t flags, void* cuda_stream);
+
+/*
  * Block-scaled contraction alone: out[M x N] = dq(a) dq(w)^T + c, fp32 output with leading dimension ldo.
  * a_codes / a_scales : M rows, w_codes / w_scales : N rows, both K-major with LATMIX_SF_TCGEN05 scales.
  * c : N fp32 or NULL.  Products of element values and power-of-two scales are exact; accumulation is fp32.

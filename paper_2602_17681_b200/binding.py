@@ -45,6 +45,7 @@ EXPORTS = {
                                              _sz, _u32, _vp]),
     "latmix_quantize_mx": (_int, [_vp, _int, _vp, _vp, _i64, _i64, _int, _int, _vp, _vp, _vp, _vp, _sz, _u32, _vp]),
     "latmix_transformation_mse": (_int, [_vp, _int, _vp, _vp, _vp, _i64, _i64, _int, _vp, _vp, _vp, _sz, _u32, _vp]),
+    "latmix_transformation_mse_block": (_int, [_vp, _int, _vp, _vp, _vp, _i64, _i64, _int, _int, _vp, _vp, _vp, _sz, _u32, _vp]),
     "latmix_mx_gemm": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _i64, _vp, _sz, _u32, _vp]),
     "latmix_linear": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _i64, _vp, _sz, _u32, _vp]),
     "latmix_linear_static": (_int, [_vp, _int, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp, _i64, _u32,
@@ -204,14 +205,19 @@ def quantize_mx(X, A, b, fmt, sf=SF_TCGEN05, dump=False, ws=None, flags=0, out=N
     return codes, scales, dumped
 
 
-def transformation_mse(X, A, b, A_inv, fmt, ws=None, flags=0):
-    """-> (E(T) as a 0-d float64 tensor, block-wise error as K/32 float64) for T(x) = x A + b; A None = identity."""
+def transformation_mse(X, A, b, A_inv, fmt, ws=None, flags=0, block=32):
+    """-> (E(T) as a 0-d float64 tensor, block-wise error as K/block float64) for T(x) = x A + b; A None = identity."""
     M, K = X.shape
-    block_err = torch.empty(K // 32, dtype=torch.float64, device=X.device)
+    block_err = torch.empty(K // block, dtype=torch.float64, device=X.device)
     mse = torch.empty((), dtype=torch.float64, device=X.device)
     ws = new_workspace(OP_TRANSFORMATION_MSE, M, K, 0, fmt, X.device) if ws is None else ws
-    _check(_lib.latmix_transformation_mse(_ptr(X), _dtype(X), _ptr(A), _ptr(b), _ptr(A_inv), M, K, fmt, _ptr(block_err), _ptr(mse),
-                                          _ptr(ws), ws.numel(), flags, _stream()), "latmix_transformation_mse")
+    if block == 32:
+        _check(_lib.latmix_transformation_mse(_ptr(X), _dtype(X), _ptr(A), _ptr(b), _ptr(A_inv), M, K, fmt, _ptr(block_err), _ptr(mse),
+                                              _ptr(ws), ws.numel(), flags, _stream()), "latmix_transformation_mse")
+    else:
+        _check(_lib.latmix_transformation_mse_block(_ptr(X), _dtype(X), _ptr(A), _ptr(b), _ptr(A_inv), M, K, fmt, block,
+                                                    _ptr(block_err), _ptr(mse), _ptr(ws), ws.numel(), flags, _stream()),
+               "latmix_transformation_mse_block")
     return mse, block_err
 
 

@@ -380,12 +380,22 @@ latmix_status_t latmix_transformation_mse(const void* X, latmix_dtype_t x_dtype,
                                           const float* A_inv, int64_t M, int64_t K, latmix_format_t fmt, double* block_err,
                                           double* mse, void* workspace, size_t workspace_bytes, uint32_t flags,
                                           void* cuda_stream) {
+    return latmix_transformation_mse_block(X, x_dtype, A, b, A_inv, M, K, fmt, 32, block_err, mse, workspace, workspace_bytes, flags,
+                                           cuda_stream);
+}
+
+latmix_status_t latmix_transformation_mse_block(const void* X, latmix_dtype_t x_dtype, const void* A, const float* b,
+                                                const float* A_inv, int64_t M, int64_t K, latmix_format_t fmt, int block,
+                                                double* block_err, double* mse, void* workspace, size_t workspace_bytes,
+                                                uint32_t flags, void* cuda_stream) {
+    if (block != 8 && block != 16 && block != 32 && block != 64 && block != 128) return LATMIX_ERR_INVALID_ARG;
     if (X == nullptr || block_err == nullptr || mse == nullptr || !valid_fmt(fmt) || !valid_dtype(x_dtype)) return LATMIX_ERR_INVALID_ARG;
     if ((A == nullptr) != (A_inv == nullptr)) return LATMIX_ERR_INVALID_ARG;        // a transform comes with its inverse
     if (fmt == LATMIX_NVFP4) return LATMIX_ERR_UNSUPPORTED;
     if (!aligned16(A_inv) || !aligned16(block_err) || (reinterpret_cast<uintptr_t>(mse) & 7u)) return LATMIX_ERR_INVALID_ARG;
     latmix_status_t s = shape_check(M, K, fmt);
     if (s != LATMIX_OK) return s;
+    if (K % block != 0) return LATMIX_ERR_SHAPE;
     size_t cb, sb;
     mx_sizes(M, K, fmt, LATMIX_SF_LINEAR, &cb, &sb);
     const size_t mk = align_up((size_t)M * (size_t)K * sizeof(float), 256);
@@ -406,7 +416,9 @@ latmix_status_t latmix_transformation_mse(const void* X, latmix_dtype_t x_dtype,
     s = latmix_quantize_mx(X, x_dtype, A, b, M, K, fmt, LATMIX_SF_LINEAR, codes, scales, D, workspace, kWorkspaceHeaderBytes, flags,
                            cuda_stream);
     if (s != LATMIX_OK) return s;
-    if (launch_dequant_diff(D, codes, scales, M, K, (int)fmt, D, st) != cudaSuccess) return LATMIX_ERR_CUDA;   // d = y - Q(y), in place
+    // d = y - Q(y), in place: from the codes the path just produced (B = 32), or re-quantised with the asked block size
+    if (block == 32) { if (launch_dequant_diff(D, codes, scales, M, K, (int)fmt, D, st) != cudaSuccess) return LATMIX_ERR_CUDA; }
+    else if (launch_quant_error_block(D, M, K, (int)fmt, block, D, st) != cudaSuccess) return LATMIX_ERR_CUDA;
     const float* err = D;                                // identity transform: the error needs no mapping back
     if (A_inv != nullptr) {
         if (!(flags & LATMIX_FLAG_FORCE_SIMT) && workspace_bytes >= need_tc && backmap_tc_supported(M, K)) {
@@ -418,7 +430,7 @@ latmix_status_t latmix_transformation_mse(const void* X, latmix_dtype_t x_dtype,
         }
         err = E;
     }
-    if (launch_block_sumsq(err, M, K, block_err, mse, st) != cudaSuccess) return LATMIX_ERR_CUDA;
+    if (launch_block_sumsq(err, M, K, block, block_err, mse, st) != cudaSuccess) return LATMIX_ERR_CUDA;
     return LATMIX_OK;
 }
 

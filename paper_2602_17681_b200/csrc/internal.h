@@ -133,7 +133,9 @@ bool backmap_tc_supported(int64_t M, int64_t K);
 size_t backmap_tc_scratch_bytes(int64_t M, int64_t K);
 cudaError_t launch_backmap_tc(const float* D, const float* A_inv, int64_t M, int64_t K, float* E, uint32_t* status,
                               void* scratch, cudaStream_t st);
-cudaError_t launch_block_sumsq(const float* E, int64_t M, int64_t K, double* block_err, double* mse, cudaStream_t st);
+cudaError_t launch_block_sumsq(const float* E, int64_t M, int64_t K, int block, double* block_err, double* mse, cudaStream_t st);
+// D = Y - Q_B(Y) for an MX block size B of 8, 16, 32, 64 or 128 (K a multiple of B); D may alias Y.
+cudaError_t launch_quant_error_block(const float* Y, int64_t M, int64_t K, int fmt, int block, float* D, cudaStream_t st);
 
 // The same for fp32 weights (both operands as three bf16 terms, nine products); K a multiple of 64.
 size_t fold_tc_f32_scratch_bytes(int64_t K, int64_t N);

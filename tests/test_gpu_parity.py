@@ -707,6 +707,53 @@ def test_transformation_mse(B, fmt, case):
     assert np.allclose(blk.cpu().numpy(), ref_blk, rtol=5e-2)
 
 
+@pytest.mark.parametrize("block", [8, 16, 64, 128])
+@pytest.mark.parametrize("fmt", [0, 1, 2])
+@pytest.mark.parametrize("case", ["full", "identity", "hadamard"])
+def test_transformation_mse_block_size_sweep(B, block, fmt, case):
+    """E(T) and E_B^i for MX block sizes other than the layer's 32 (the block-size sweep of the numerical analysis in
+    Sec. 3.1): against the oracle's quantiser with that block size, on the kernel's own transformed values (tight) and on
+    the all-fp64 chain (loose: near-ties)."""
+    name = H.FMT_NAME[fmt]
+    M, K = 200, 384
+    X = synth.make_activations(M, K, 53, dtype="bf16")
+    flags = 0
+    if case == "identity":
+        A = A_inv = None
+        b = (torch.randn(K) * 0.1).float()
+    elif case == "hadamard":
+        A, b, A_inv = synth.make_block_transform(K, 53, "hadamard")
+        flags = B.FLAG_BLOCK_DIAG
+    else:
+        A, b, A_inv = synth.make_transform(K, 53, "bf16")
+    d = lambda t: None if t is None else t.cuda()
+    mse, blk = B.transformation_mse(X.cuda(), d(A), d(b), d(A_inv), fmt, flags=flags, block=block)
+    assert blk.numel() == K // block
+    _, _, Y = B.quantize_mx(X.cuda(), d(A), d(b), fmt, B.SF_LINEAR, dump=True, flags=flags)
+    Yg = Y.double().cpu().numpy()
+    qc, qs = orc.mx_quantize(Yg, name, block=block)
+    e = Yg - orc.mx_dequantize(qc, qs, name, block=block)
+    if A_inv is not None:
+        e = e @ A_inv.double().numpy()
+    want = (e ** 2).reshape(M, K // block, block).mean(axis=(0, 2))
+    assert np.allclose(blk.cpu().numpy(), want, rtol=2e-5, atol=0)
+    assert np.isclose(float(mse), (e ** 2).mean(), rtol=2e-5, atol=0)
+    X64 = X.double().numpy()
+    b64 = None if b is None else b.double().numpy()
+    if case == "identity":
+        ref_mse, _ = orc.transformation_mse(X64, None, None, b64, name, block=block)
+    elif case == "hadamard":
+        dense = np.kron(np.eye(K // 32), orc.hadamard_block(32))
+        ref_mse, _ = orc.transformation_mse(X64, dense, A_inv.double().numpy(), b64, name, block=block)
+    else:
+        ref_mse, _ = orc.transformation_mse(X64, A.double().numpy(), A_inv.double().numpy(), b64, name, block=block)
+    # Hadamard blocks of bf16 inputs put many values exactly on rounding boundaries, where fp32 and fp64 sums part ways
+    assert np.isclose(float(mse), ref_mse, rtol=3e-2)
+    with pytest.raises(B.LatmixError) as err:
+        B.transformation_mse(X.cuda(), d(A), d(b), d(A_inv), fmt, flags=flags, block=24)
+    assert err.value.code == B.ERR_INVALID_ARG
+
+
 def test_transformation_mse_is_reproducible_and_checks_arguments(B):
     M, K, fmt = 128, 256, 0
     X = synth.make_activations(M, K, 52, dtype="bf16")
