@@ -109,6 +109,7 @@ mx_gemm_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
     grid_dependency_wait();            // set-up above may have overlapped the previous kernel; its results are needed from here on
+    grid_launch_dependents();          // the kernel after this one may set itself up on SMs this one has left
     const int num_tiles = p.m_tiles * p.n_tiles;
     const int pair = (int)cluster_id_x(), num_pairs = (int)num_clusters_x();
     constexpr uint16_t kBoth = 3, kLeader = 1;

@@ -116,6 +116,8 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
     grid_launch_dependents();          // a product kernel launched for it may set itself up on SMs this kernel has left
+    grid_dependency_wait();            // and this one may have been set up while its predecessor still ran: its results (the
+                                       // activations) are read, and its operands (the codes of the step before) overwritten, from here on
     const int pair = (int)cluster_id_x(), num_pairs = (int)num_clusters_x();
     constexpr uint16_t kBoth = 3;
 
@@ -367,7 +369,13 @@ cudaError_t launch_transform_quant_pair_tc(const TransformQuantArgs& a, cudaStre
     p.num_items = split ? tiles + rem : tiles;
     const unsigned grid = 2u * (unsigned)(p.num_items < pairs ? p.num_items : pairs);
     void* args[] = {(void*)&tm_x, (void*)&tm_a, (void*)&p};
-    e = cudaLaunchKernel(kern, dim3(grid), dim3(THREADS), args, SMEM_BYTES, st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;      // the kernel waits for its predecessor itself, after its set-up
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelExC(&cfg, kern, args);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
 }

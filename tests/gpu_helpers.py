@@ -105,16 +105,17 @@ K_PER_MMA = {"mxfp4": 64, "mxfp8": 32, "mxint4": 32, "mxint8": 16}      # MXINT8
 def block_scaled_unit(K, fmt_name, simt=False):
     """Relative size of the accumulation error of the block-scaled product, per unit of sum |dq(a)||dq(w)|.
 
-    Products of element values and power-of-two scales are exact.  On the tensor cores the fp32 accumulator is
-    rounded once per MMA instruction, K / k_per_mma times, each time by at most 2^-24 of a partial sum that never exceeds
-    sum |a||w|; four more roundings cover the sum inside one instruction.  The CUDA-core kernel adds one 32-term fp32
-    FMA chain per block and then K/32 block sums across 32 lanes and a five-step shuffle tree.
-    This is a worst-case bound (every rounding in the same direction on same-sign data).  Measured on B200 with random
-    codes and scales spread over 2^+-6 the largest error is 7 to 12 units of 2^-24 where the bound is 20 to 36 (K = 1024
-    to 2048, MXFP4); on layer data, whose products cancel, it is below 1 unit."""
+    Products of element values and power-of-two scales are exact.  On the tensor cores the products of one MMA
+    instruction are aligned to the largest exponent among them and added to the fp32 accumulator with truncation, so an
+    instruction can lose up to 2^-23 of a partial sum that never exceeds sum |a||w|; there are K / k_per_mma instructions,
+    and four more units cover the sum inside one instruction.  The CUDA-core kernel adds one 32-term fp32 FMA chain per
+    block and then K/32 block sums across 32 lanes and a five-step shuffle tree.
+    This is a worst-case bound.  Measured on B200 with random codes and block scales spread over 2^+-6 the largest error is
+    7 to 15 units of 2^-24 where the bound is 24 to 72 (K = 256 to 2048; a bound of one 2^-24 per instruction was exceeded
+    by 7 of 15.7 million elements at K = 256, MXFP8); on layer data, whose products cancel, it stays below 1 unit."""
     if simt:
         return (32 + K / 1024.0 + 6.0) * 2.0 ** -24
-    return (K / K_PER_MMA[fmt_name] + 4.0) * 2.0 ** -24
+    return (K / K_PER_MMA[fmt_name] + 4.0) * 2.0 ** -23
 
 
 def gemm_error_ratio(out, ref, a_codes, a_scales, w_codes, w_scales, fmt_name, c=None):
