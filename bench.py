@@ -36,7 +36,7 @@ FMT_RATIO_TO_BF16 = {"mxfp4": 4.0, "mxfp8": 2.0, "mxint8": 1.0, "mxint4": 2.0}  
 METRIC = "fused transform+MX linear throughput"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from an ncu capture of this command
 # with the kernel as it is now; None = not captured (or the kernel has changed since the counters were taken).
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_gate_up": None}
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg2_gate_up": 219.0e6}
 
 
 def load_peaks():
@@ -341,7 +341,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     k2_tflops = f3 / (t_k2 * 1e-3) / 1e12
     p_mx = bf16[regime_k] * ratio
     if M > 128:
-        kernel = "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)" if cfg.fmt == "mxint8" else "mx_gemm_pair_tc_kernel (block-scaled GEMM)"
+        kernel = "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)" if cfg.fmt == "mxint8" else "mx_gemm_wide_tc_kernel (block-scaled GEMM, 256 x 256 CTA-pair tiles)"
     elif cfg.fmt == "mxint8":
         kernel = "mxint8_gemm_decode_tc_kernel (int8 -> bf16 in shared memory)" if M <= 16 else "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)"
     else:
