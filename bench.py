@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2602_17681_b200 import synth  # noqa: E402
 
-FMT_RATIO_TO_BF16 = {"mxfp4": 4.0, "mxfp8": 2.0, "mxint8": 1.0, "mxint4": 2.0}   # nominal dense tensor-rate ratios on B200
+FMT_RATIO_TO_BF16 = {"mxfp4": 4.0, "mxfp8": 2.0, "mxint8": 1.0, "mxint4": 2.0, "nvfp4": 4.0}   # nominal dense tensor-rate ratios on B200
 METRIC = "fused transform+MX linear throughput"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from an ncu capture of this command
 # with the kernel as it is now; None = not captured (or the kernel has changed since the counters were taken).
@@ -66,9 +66,10 @@ def layer_flops(M, K, N, transform="full"):
 
 
 def layer_bytes(M, K, N, fmt, transform="full"):
-    code = 0.5 if fmt == "mxfp4" else 1.0
+    code = 0.5 if fmt in ("mxfp4", "nvfp4") else 1.0
+    scale = 1 / 16.0 if fmt == "nvfp4" else 1 / 32.0
     a_bytes = 2.0 * K * K if transform == "full" else 2.0 * K * 32
-    return 2.0 * M * K + a_bytes + N * K * code + N * K / 32.0 + 4.0 * M * N
+    return 2.0 * M * K + a_bytes + N * K * (code + scale) + 4.0 * M * N
 
 
 def shard_rows(M_total, rank, world):
@@ -196,7 +197,7 @@ def run_reference(args, cfg, rank, world):
 
 
 def workload_name(cfg):
-    return f"{cfg.name}: X {cfg.M}x{cfg.K} {cfg.x_dtype}, A {cfg.K}x{cfg.K}, W {cfg.K}x{cfg.N}, {cfg.fmt} block 32"
+    return f"{cfg.name}: X {cfg.M}x{cfg.K} {cfg.x_dtype}, A {cfg.K}x{cfg.K}, W {cfg.K}x{cfg.N}, {cfg.fmt} block {16 if cfg.fmt == 'nvfp4' else 32}"
 
 
 # ----------------------------------------------------------------------------------------------------
@@ -219,8 +220,14 @@ def run_ours(args, cfg, rank, world, local_rank):
         blocks, _, A_inv = synth.make_block_transform(K, cfg.seed, "hadamard", a_dtype=cfg.x_dtype, device=dev)
         layer["A"], layer["A_inv"], layer["b"] = blocks, A_inv, torch.zeros(K, dtype=torch.float32, device=dev)
         flags = B.FLAG_BLOCK_DIAG
+    g_w = g_a = None
+    if cfg.fmt == "nvfp4":
+        # the two tensor scales are inputs of the format: calibrated here, at set-up, as max|.| / (448 * 6) of the folded weights
+        # and of the transformed activations of the first input set (plain torch products; not part of the timed path)
+        g_w = float((layer["A_inv"] @ layer["W"].float()).abs().max()) / (448.0 * 6.0)
+        g_a = float((layer["X"].float() @ layer["A"].float() + layer["b"]).abs().max()) * 1.25 / (448.0 * 6.0)
     t0 = time.perf_counter()
-    Wq, Wsc, c, _ = B.fold_weights(layer["A_inv"], layer["b"], layer["W"], layer["bias"], fmt)
+    Wq, Wsc, c, _ = B.fold_weights(layer["A_inv"], layer["b"], layer["W"], layer["bias"], fmt, tensor_scale=g_w)
     torch.cuda.synchronize()
     fold_ms = (time.perf_counter() - t0) * 1e3
     sets = []
@@ -230,6 +237,8 @@ def run_ours(args, cfg, rank, world, local_rank):
         sets.append(dict(X=X, A=layer["A"].clone(), b=layer["b"].clone(), Wq=Wq.clone(), Wsc=Wsc.clone(), c=c.clone(),
                          out=torch.empty(M, N, dtype=torch.float32, device=dev)))
     ws = B.new_workspace(B.OP_LINEAR, M, K, N, fmt, dev)
+    if g_a is not None:
+        B.workspace_set_tensor_scale(ws, g_a)
 
     def step(i):
         s = sets[i % n_sets]
@@ -287,6 +296,8 @@ def run_ours(args, cfg, rank, world, local_rank):
 
     # ---- per-kernel breakdown: the same two kernels, launched through the two half-calls, events around each
     a_codes, a_scales = B.alloc_mx(M, K, fmt, B.SF_TCGEN05, dev)
+    if g_a is not None:
+        B.set_tensor_scale(a_scales, M, K, fmt, B.SF_TCGEN05, g_a)
     k_iters = max(10, min(args.steps, 200))
     sampler_k = ClockSampler(local_rank)
     sampler_k.start()
@@ -332,7 +343,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         if args.transform == "full":
             t1_s = f1 / (p_bf16 * 1e12)
         else:   # the block-wise transform is bound by reading X and writing codes and scales
-            t1_s = (2.0 * M * K + M * K * ((0.5 if cfg.fmt == "mxfp4" else 1.0) + 1 / 32.0)) / (peaks["hbm_gbs"] * 1e9)
+            t1_s = (2.0 * M * K + M * K * ((0.5 if cfg.fmt in ("mxfp4", "nvfp4") else 1.0) + 1 / 32.0)) / (peaks["hbm_gbs"] * 1e9)
         r2 = max(t1_s + f3 / (p_bf16 * ratio * 1e12), hbm_s) * 1e3
         r1 = max((f1 + f3) / (p_bf16 * ratio * 1e12), hbm_s) * 1e3
         return r2, r1
@@ -368,13 +379,13 @@ def run_ours(args, cfg, rank, world, local_rank):
                     "mx_gemm_ms": t_k2, "mx_gemm_tflops": k2_tflops},
     }
     if pipe is not None:
-        own = {"mxfp4": "mxf4", "mxfp8": "mxf8", "mxint4": "mxf8", "mxint8": "bf16"}[cfg.fmt]
+        own = {"mxfp4": "mxf4", "nvfp4": "mxf4", "mxfp8": "mxf8", "mxint4": "mxf8", "mxint8": "bf16"}[cfg.fmt]
         roofline["pipe_probe"] = {"tflops": pipe, "frac_of_probe": k2_tflops / pipe[own], "kind": own,
                                   "note": "back-to-back tcgen05.mma 128 x 256 on shared-memory operands, every SM, about 2 ms "
                                           "per kind, at the clock the probe itself ran at"}
     if M <= 64:
         # small batches: the dominant kernel streams the weights once; algorithmic bytes = codes + scales of both operands + result
-        code = 0.5 if cfg.fmt == "mxfp4" else 1.0
+        code = 0.5 if cfg.fmt in ("mxfp4", "nvfp4") else 1.0
         k2_bytes = (N + M) * K * (code + 1 / 32.0) + 4.0 * M * N
         gbs = k2_bytes / (t_k2 * 1e-3) / 1e9
         roofline.update({"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
@@ -396,6 +407,8 @@ def run_ours(args, cfg, rank, world, local_rank):
             slots.append(dict(stream=torch.cuda.Stream(device=dev), dX=torch.empty_like(sets[0]["X"]),
                               dout=sets[i]["out"], hout=torch.empty(M, N, dtype=torch.float32).pin_memory(),
                               ws=ws if i == 0 else B.new_workspace(B.OP_LINEAR, M, K, N, fmt, dev)))
+            if g_a is not None:
+                B.workspace_set_tensor_scale(slots[-1]["ws"], g_a)
         torch.cuda.synchronize()
         n_e2e = max(4, min(args.steps, 10))
 
@@ -432,7 +445,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         e2e = {"value": world * (f1 + f3) / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": hX.numel() * hX.element_size(), "d2h_bytes_per_step": hout.numel() * 4}
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.transform == "full":
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.transform == "full" and cfg.fmt != "nvfp4":
         rows, cols = 1024, 4096
         tf, sec = time_oracle(cfg, rows, cols, steps=5, warmup=1)
         cpu_baseline = {"value": tf, "unit": "TFLOP/s", "cores": oracle_threads(), "kind": "oracle",
@@ -444,7 +457,8 @@ def run_ours(args, cfg, rank, world, local_rank):
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {"mxfp4": "fp4(e2m1)+e8m0 x bf16 transform", "mxfp8": "fp8(e4m3)+e8m0 x bf16 transform",
-                      "mxint8": "int8+e8m0 x bf16 transform", "mxint4": "int4 (as e4m3 bytes)+e8m0 x bf16 transform"}[cfg.fmt],
+                      "mxint8": "int8+e8m0 x bf16 transform", "mxint4": "int4 (as e4m3 bytes)+e8m0 x bf16 transform",
+                      "nvfp4": "fp4(e2m1)+e4m3 per 16+fp32 tensor scale x bf16 transform"}[cfg.fmt],
             "data": "synthetic",
             "config": {"workload": workload_name(cfg) + (", online transform: 32x32 Hadamard blocks (T3)" if args.transform == "blockdiag" else ""),
                        "rows_per_gpu": M, "parallelism": f"rows x{world} (replicated weights, no collective)",

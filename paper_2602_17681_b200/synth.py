@@ -25,7 +25,7 @@ class LayerConfig:
     M: int
     K: int
     N: int
-    fmt: str = "mxfp4"            # mxfp4 | mxfp8 | mxint8
+    fmt: str = "mxfp4"            # mxfp4 | mxfp8 | mxint8 | mxint4 | nvfp4
     x_dtype: str = "bf16"         # bf16 | f32
     act: str = "normal"           # normal | student_t3
     outlier_frac: float = 0.01    # fraction of channels scaled up (or an absolute count if >= 1)
@@ -44,6 +44,7 @@ CONFIGS = {
     "cfg2_gate_up_fused": LayerConfig("cfg2_gate_up_fused", 4096, 4096, 28672, seed=2),
     "cfg2_down": LayerConfig("cfg2_down", 4096, 14336, 4096, seed=2),
     "cfg2_gate_up_int4": LayerConfig("cfg2_gate_up_int4", 4096, 4096, 14336, fmt="mxint4", seed=2),
+    "cfg2_gate_up_nvfp4": LayerConfig("cfg2_gate_up_nvfp4", 4096, 4096, 14336, fmt="nvfp4", seed=2),
     "cfg3_fp8_m1": LayerConfig("cfg3_fp8_m1", 1, 4096, 14336, fmt="mxfp8", seed=3),
     "cfg3_fp8_m16": LayerConfig("cfg3_fp8_m16", 16, 4096, 14336, fmt="mxfp8", seed=3),
     "cfg3_fp8_m8192": LayerConfig("cfg3_fp8_m8192", 8192, 4096, 14336, fmt="mxfp8", seed=3),
