@@ -49,7 +49,9 @@ constexpr int STAGE_BYTES = SLABS * (A_BYTES + B_BOXES * B_BOX_BYTES);    // 64 
 constexpr int STAGES = 3;
 constexpr int NUM_ACC = 2;
 constexpr int BAR_BYTES = 1024;
-constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + BAR_BYTES;
+constexpr int CODE_STAGING_BYTES = 4 * 32 * BLOCK_N;            // per epilogue warp: 32 rows x up to 256 code bytes (8-bit formats)
+constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + BAR_BYTES + CODE_STAGING_BYTES;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr int TMEM_COLS = 512;
 constexpr int THREADS = 6 * 32;
 }  // namespace tqp
@@ -99,6 +101,7 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + NUM_ACC + a); };   // leader: 4 warps x 2 CTAs
     const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 2 * NUM_ACC);
+    const uint32_t code_staging_base = bar_base + BAR_BYTES;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
     const int warp_idx = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -233,6 +236,18 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
         // ------------------------------------------------------------------ quantising epilogue (warps 2..5, both CTAs)
         const int q = warp_idx & 3;                                  // tensor-memory lane quarter this warp may read
         constexpr int kRMax = FormatTraits<FMT == FMT_NVFP4 ? FMT_FP4 : FMT>::kRMax;
+        // The codes of a tile go out through shared memory: a thread owns one row (32 values per chunk, i.e. 16 or 32 code
+        // bytes), so stored directly a warp's instruction would touch 32 rows with 16 bytes each.  Staged (16-byte pieces,
+        // piece index XOR row to keep the banks apart), a warp then writes whole rows: 8 or 16 lanes per row, 128 or 256
+        // contiguous bytes.
+        constexpr bool kPacked = FMT == FMT_FP4 || FMT == FMT_NVFP4;          // two codes per byte
+        constexpr int kPiecesPerChunk = kPacked ? 1 : 2;                      // 16-byte pieces of codes per thread and chunk
+        constexpr int kRowBytes = kPacked ? BLOCK_N / 2 : BLOCK_N;            // staging row pitch
+        const uint32_t stg = code_staging_base + (uint32_t)(warp_idx - 2) * (32 * BLOCK_N);
+        auto stage_piece = [&](int piece, const uint4& w) {
+            const uint32_t dst = stg + (uint32_t)lane * kRowBytes + (uint32_t)(((piece & ~7) | ((piece ^ lane) & 7)) * 16);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
+        };
         float nv_g = 1.0f;                                           // NVFP4: the tensor scale, from the scale buffer's trailer
         if (FMT == FMT_NVFP4 && p.codes != nullptr) nv_g = *nvfp4_tensor_scale_ptr(p.scales, p.M, p.K, p.sf_layout);
         uint32_t item_count = 0;
@@ -280,7 +295,7 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
                     uint2 w0, w1;
                     const uint32_t s0 = nvfp4_quantize_block(v, nv_g, w0), s1 = nvfp4_quantize_block(v + 16, nv_g, w1);
                     if (blk_ok) {
-                        *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (col0 >> 1)) = make_uint4(w0.x, w0.y, w1.x, w1.y);
+                        stage_piece(chunk, make_uint4(w0.x, w0.y, w1.x, w1.y));
                         const int64_t kblk = col0 >> 4;
                         const size_t off = p.sf_layout == LATMIX_SF_LINEAR ? (size_t)(row * (p.K >> 4) + kblk)
                                                                            : sf_tcgen05_offset(row, kblk, p.sf_kt_total);
@@ -294,14 +309,12 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
                 for (int i = 0; i < 32; ++i) v[i] = (v[i] * f.x) * f.y;
                 if (blk_ok) {
                     if (FMT == FMT_FP4 || FMT == FMT_NVFP4) {
-                        uint4 w = make_uint4(pack8_fp4(v), pack8_fp4(v + 8), pack8_fp4(v + 16), pack8_fp4(v + 24));
-                        *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (col0 >> 1)) = w;
+                        stage_piece(chunk, make_uint4(pack8_fp4(v), pack8_fp4(v + 8), pack8_fp4(v + 16), pack8_fp4(v + 24)));
                     } else {
                         uint2 w0, w1, w2, w3;
                         w0 = pack8_bytes<FMT>(v); w1 = pack8_bytes<FMT>(v + 8); w2 = pack8_bytes<FMT>(v + 16); w3 = pack8_bytes<FMT>(v + 24);
-                        uint4* d = reinterpret_cast<uint4*>(p.codes + row * (int64_t)p.K + col0);
-                        d[0] = make_uint4(w0.x, w0.y, w1.x, w1.y);
-                        d[1] = make_uint4(w2.x, w2.y, w3.x, w3.y);
+                        stage_piece(2 * chunk, make_uint4(w0.x, w0.y, w1.x, w1.y));
+                        stage_piece(2 * chunk + 1, make_uint4(w2.x, w2.y, w3.x, w3.y));
                     }
                     const int64_t kblk = col0 >> 5;
                     if (p.sf_layout == LATMIX_SF_LINEAR) {
@@ -320,6 +333,24 @@ transform_quant_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const _
             if (lane == 0) {                                      // this warp has drained its quarter of the accumulator
                 if (leader) mbar_arrive(tempty_bar(acc));
                 else mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
+            }
+            if (p.codes != nullptr) {
+                // the staged codes, whole rows at a time: `lanes_per_row` lanes write one row's 16-byte pieces side by side
+                const int pieces = (bn >> 5) * kPiecesPerChunk;                  // per row in this item: 4, 8 or 16
+                const int rows_per_it = 32 / pieces, piece = lane % pieces;
+                const int64_t row_base = m0 + (int)rank * BLOCK_M + q * 32;
+                const int64_t row_pitch = kPacked ? (int64_t)(p.K >> 1) : (int64_t)p.K, col_byte0 = kPacked ? (n0 >> 1) : n0;
+                for (int r0 = 0; r0 < 32; r0 += rows_per_it) {
+                    const int r = r0 + lane / pieces;
+                    const uint32_t src = stg + (uint32_t)r * kRowBytes + (uint32_t)(((piece & ~7) | ((piece ^ r) & 7)) * 16);
+                    uint4 w;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "r"(src));
+                    // a piece = 32 elements (4-bit) or 16 (8-bit); K is a multiple of 32, so a piece is inside the matrix or outside it
+                    const int64_t elem0 = n0 + (int64_t)piece * (kPacked ? 32 : 16);
+                    if (row_base + r < p.M && elem0 < p.K)
+                        *reinterpret_cast<uint4*>(p.codes + (row_base + r) * row_pitch + col_byte0 + piece * 16) = w;
+                }
+                __syncwarp();                                     // the buffer is rewritten by the next item's first chunk
             }
         }
     }
