@@ -510,3 +510,34 @@ def test_mxint4_reading_by_hand():
     assert orc.mx_dequantize(codes, scales, "mxint4", 4).tolist() == [[10.0, 0.0, -4.0, 0.0]]
     codes, scales = orc.mx_quantize(np.array([[7.9, -7.6]]), "mxint4", block=2)
     assert codes.tolist() == [[7, 9]] and scales.tolist() == [[127]]
+
+
+# ---------------------------------------------------------------- other block sizes (the block-size sweep of Sec. 3.1)
+@pytest.mark.parametrize("block", [8, 16, 64, 128])
+@pytest.mark.parametrize("fmt", OCP_FMTS)
+def test_other_block_sizes_brute_force_and_invariants(fmt, block):
+    """Eq. q_mx with a block size other than 32, as the sweep over block sizes uses it: whole blocks against the
+    exact-rational brute force, the floor rule of the scale, values on grid x 2^E; and the transformation MSE with a
+    block as long as the row equals a plain per-row quantisation error."""
+    f = orc.FORMATS[fmt]
+    rng = np.random.default_rng(40 + block)
+    Y = rng.standard_normal((6, 2 * block)) * np.exp(rng.standard_normal((6, 1)) * 3)
+    Y[:, 3] *= 40
+    codes, sb = orc.mx_quantize(Y, fmt, block=block)
+    for r in range(6):
+        for i in range(2):
+            want_codes, want_sb = orc.mx_quantize_block_exact(Y[r, i * block:(i + 1) * block], fmt)
+            assert codes[r, i * block:(i + 1) * block].tolist() == want_codes and int(sb[r, i]) == want_sb
+    dq = orc.mx_dequantize(codes, sb, fmt, block=block)
+    s = np.ldexp(1.0, sb.astype(np.int64) - 127)
+    amax = np.abs(Y).reshape(6, 2, block).max(2)
+    assert np.all(s <= amax * 2.0 ** -f.r_max) and np.all(amax * 2.0 ** -f.r_max < 2 * s)
+    assert np.all(np.isin(np.abs(dq).reshape(6, 2, block) / s[:, :, None], f.grid))
+    # identity transform: E(T) is the mean squared quantisation error, block by block
+    mse, per_block = orc.transformation_mse(Y, None, None, None, fmt, block=block)
+    want = ((Y - dq) ** 2).reshape(6, 2, block).mean(axis=(0, 2))
+    assert np.allclose(per_block, want, rtol=1e-13) and math.isclose(mse, want.mean(), rel_tol=1e-13)
+    # a coarser block never has a smaller scale than the finer blocks it contains
+    if block >= 16:
+        _, sb_fine = orc.mx_quantize(Y, fmt, block=block // 2)
+        assert np.all(sb == sb_fine.reshape(6, 2, 2).max(2))
