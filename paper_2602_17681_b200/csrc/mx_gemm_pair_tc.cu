@@ -21,8 +21,10 @@
 //             bytes).  That commit hop runs beside the TMA latency of the code tiles, not after it.
 //   warp 1    leader: per K slab one wait, four tcgen05.mma.cta_group::2 .block_scale, one commit.  The loop is
 //             unrolled over the stages and every operand is computed once, before the loop.
-//   warps 4-7 epilogue (both CTAs): tcgen05.ld, + c[n], swizzled staging, TMA store; one arrival per warp on the
-//             leader's "accumulator empty" barrier (remote for the peer).
+//   warps 4-7 epilogue (both CTAs): the tile's c[n] fetched into shared memory before the wait; the accumulator read in
+//             two batches of three tcgen05.ld issued together (one at a time they made the epilogue the slowest part:
+//             a load takes about 2000 cycles while MMAs run); + c, swizzled staging, TMA store; one arrival per warp on
+//             the leader's "accumulator empty" barrier (remote for the peer) after the last batch has been read.
 // Every wait is bounded; whatever happens, all threads of both CTAs meet at a cluster barrier before tensor
 // memory is released and the CTAs exit, so neither CTA can touch a peer that has already gone.
 #include "internal.h"
@@ -49,8 +51,9 @@ struct MxGemmPairCfg {
     static constexpr int STAGES = 5;                               // code ring; the issue loops are unrolled over it
     static constexpr int SF_SLOTS = 8;                             // scale ring in shared memory
     static constexpr int STAGING_BYTES = 4 * STG_BUFS * 4096;      // per epilogue warp: 32 rows x 128 bytes
+    static constexpr int CVEC_BYTES = 4 * BLOCK_N * 4;              // each epilogue warp's copy of the tile's c[n]
     static constexpr int BAR_BYTES = 1024;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + SF_SLOTS * SF_SLOT_BYTES + STAGING_BYTES + BAR_BYTES;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + SF_SLOTS * SF_SLOT_BYTES + STAGING_BYTES + CVEC_BYTES + BAR_BYTES;
     static constexpr int ACC_COLS = NUM_ACC * BLOCK_N;
     static constexpr int SF_COLS = SF_KT * 4 + SF_KT * NB_RT * 4;  // tensor-memory columns of one K slab's scales
     static constexpr int TMEM_COLS = 512;
@@ -83,7 +86,8 @@ mx_gemm_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sf_base = smem_base + STAGES * Cfg::STAGE_BYTES;
     const uint32_t staging_base = sf_base + Cfg::SF_SLOTS * Cfg::SF_SLOT_BYTES;
-    const uint32_t bar_base = staging_base + Cfg::STAGING_BYTES;
+    const uint32_t cvec_base = staging_base + Cfg::STAGING_BYTES;
+    const uint32_t bar_base = cvec_base + Cfg::CVEC_BYTES;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };      // leader: both CTAs' code bytes landed AND scales copied
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };           // each CTA: stage may be refilled
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
@@ -248,54 +252,85 @@ mx_gemm_pair_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
         // ------------------------------------------------------------------ epilogue (warps 4..7, both CTAs)
         const int q = warp_idx & 3;                     // tensor-memory lane quarter this warp may read
         const uint32_t stg0 = staging_base + (uint32_t)(warp_idx - 4) * STG_BUFS * 4096u;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t cvec = cvec_base + (uint32_t)(warp_idx - 4) * (BLOCK_N * 4);
         uint32_t tile_count = 0, stg_it = 0;
+        int tile_n0 = 0;
         bool ok = true;
+        // one 32 x 32 piece of the result: + c, into the swizzled staging buffer, out through the copy engine
+        auto store_chunk = [&](const uint32_t (&r)[32], int row0, int col0) {
+            const uint32_t stg = stg0 + (stg_it % STG_BUFS) * 4096u;
+            ++stg_it;
+            if (lane == 0) bulk_wait_read<STG_BUFS - 1>();       // the store that last used this buffer has read it
+            __syncwarp();
+            const uint32_t cv_addr = cvec + (uint32_t)(col0 - tile_n0) * 4u;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {                        // 128-byte swizzle: chunk t of row `lane` -> t ^ (lane & 7)
+                float cv[4];                                     // every lane reads the same address: a broadcast
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cv[0]), "=f"(cv[1]), "=f"(cv[2]), "=f"(cv[3]) : "r"(cv_addr + 16u * t));
+                const float4 v = make_float4(__uint_as_float(r[4 * t]) + cv[0], __uint_as_float(r[4 * t + 1]) + cv[1],
+                                             __uint_as_float(r[4 * t + 2]) + cv[2], __uint_as_float(r[4 * t + 3]) + cv[3]);
+                const uint32_t dst = stg + (uint32_t)lane * 128u + (uint32_t)((t ^ (lane & 7)) * 16);
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && col0 < p.N && row0 < p.M) {
+                tma_store_2d(&tm_out, stg, col0, row0);
+                bulk_commit();
+            }
+        };
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++tile_count) {
             const int m0 = (tile % p.m_tiles) * 256 + (int)rank * Cfg::BLOCK_M, n0 = (tile / p.m_tiles) * BLOCK_N;
             const uint32_t acc = tile_count % NUM_ACC, acc_ph = (tile_count / NUM_ACC) & 1u;
+            // the tile's values of c into this warp's shared-memory copy while the MMAs still run (a lane brings eight of them);
+            // the previous tile's last reads of the copy lie before the __syncwarp of its last chunk
+            tile_n0 = n0;
+            if (lane * 8 < BLOCK_N) {
+                float4 c0 = make_float4(0.f, 0.f, 0.f, 0.f), c1 = c0;
+                const int cn = n0 + lane * 8;
+                if (p.c != nullptr) {
+                    if (cn + 8 <= p.N) {
+                        c0 = __ldg(reinterpret_cast<const float4*>(p.c + cn));
+                        c1 = __ldg(reinterpret_cast<const float4*>(p.c + cn) + 1);
+                    } else {
+                        float t[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) t[i] = cn + i < p.N ? p.c[cn + i] : 0.f;
+                        c0 = make_float4(t[0], t[1], t[2], t[3]); c1 = make_float4(t[4], t[5], t[6], t[7]);
+                    }
+                }
+                const uint32_t dst = cvec + (uint32_t)lane * 32u;
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(c0.x), "f"(c0.y), "f"(c0.z), "f"(c0.w) : "memory");
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + 16u), "f"(c1.x), "f"(c1.y), "f"(c1.z), "f"(c1.w) : "memory");
+            }
+            __syncwarp();
             ok = mbar_wait(tfull_bar(acc), acc_ph, p.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            // The accumulator leaves in batches of three 32-column loads issued together: a tcgen05.ld takes far longer
+            // while MMAs run (about 2000 cycles against 100 on an idle pipe) but several overlap.  After the last batch the
+            // buffer goes back to the MMA warp, before this warp's stores.
+            const int row0 = m0 + q * 32;
+            const uint32_t t0 = lane_base + acc * BLOCK_N;
+            constexpr int kBatches = BLOCK_N / 96;
+            static_assert(BLOCK_N % 96 == 0, "the epilogue reads the accumulator in batches of 96 columns");
 #pragma unroll 1
-            for (int chunk = 0; chunk < BLOCK_N / 32; ++chunk, ++stg_it) {
-                uint32_t r[32];
-                tc_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BLOCK_N + chunk * 32, r);
+            for (int bt = 0; bt < kBatches; ++bt) {
+                uint32_t r0[32], r1[32], r2[32];
+                tc_ld_32x32b_x32(t0 + bt * 96u, r0); tc_ld_32x32b_x32(t0 + bt * 96u + 32u, r1); tc_ld_32x32b_x32(t0 + bt * 96u + 64u, r2);
                 tc_wait_ld();
-                const int col0 = n0 + chunk * 32;
-                const uint32_t stg = stg0 + (stg_it % STG_BUFS) * 4096u;
-                if (lane == 0) bulk_wait_read<STG_BUFS - 1>();   // the store that last used this buffer has read it
-                __syncwarp();
-                float cv[32];
-                if (p.c != nullptr && col0 + 32 <= p.N) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float4 t = __ldg(reinterpret_cast<const float4*>(p.c + col0) + j);
-                        cv[4 * j] = t.x; cv[4 * j + 1] = t.y; cv[4 * j + 2] = t.z; cv[4 * j + 3] = t.w;
+                if (bt == kBatches - 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {                              // this warp has drained its quarter of the accumulator
+                        if (leader) mbar_arrive(tempty_bar(acc));
+                        else mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
                     }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) cv[i] = (p.c != nullptr && col0 + i < p.N) ? p.c[col0 + i] : 0.f;
                 }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {                     // 128-byte swizzle: chunk j of row `lane` -> j ^ (lane & 7)
-                    const float4 v = make_float4(__uint_as_float(r[4 * j]) + cv[4 * j], __uint_as_float(r[4 * j + 1]) + cv[4 * j + 1],
-                                                 __uint_as_float(r[4 * j + 2]) + cv[4 * j + 2], __uint_as_float(r[4 * j + 3]) + cv[4 * j + 3]);
-                    const uint32_t dst = stg + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) * 16);
-                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0 && col0 < p.N && m0 + q * 32 < p.M) {
-                    tma_store_2d(&tm_out, stg, col0, m0 + q * 32);
-                    bulk_commit();
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {                                      // this warp has drained its quarter of the accumulator
-                if (leader) mbar_arrive(tempty_bar(acc));
-                else mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
+                const int c0 = n0 + bt * 96;
+                store_chunk(r0, row0, c0); store_chunk(r1, row0, c0 + 32); store_chunk(r2, row0, c0 + 64);
             }
         }
         if (lane == 0) bulk_wait<0>();
