@@ -214,9 +214,7 @@ static cudaError_t launch_bd_mma_variant(const QuantArgs& a, const void* A_block
 }
 
 cudaError_t launch_blockdiag_quant_mma(const QuantArgs& a, const void* A_blocks, cudaStream_t st) {
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     cudaError_t e;
     if (a.fmt == FMT_FP4) e = launch_bd_mma_variant<FMT_FP4>(a, A_blocks, sms, st);
     else if (a.fmt == FMT_FP8) e = launch_bd_mma_variant<FMT_FP8>(a, A_blocks, sms, st);

@@ -256,9 +256,7 @@ cudaError_t launch_mxint8_gemm_tc(const MxGemmArgs& a, void* scratch, cudaStream
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     __nv_bfloat16* a16 = static_cast<__nv_bfloat16*>(scratch);
     __nv_bfloat16* w16 = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(scratch) + up((size_t)a.M * (size_t)a.K * 2));
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     auto blocks = [&](int64_t rows) {                       // a warp per row at a time, at most 8 CTAs of 8 warps per SM
         const int64_t want = (rows + 7) / 8;
         return (unsigned)(want < (int64_t)sms * 8 ? (want > 0 ? want : 1) : (int64_t)sms * 8);
@@ -280,7 +278,7 @@ cudaError_t launch_mxint8_gemm_tc(const MxGemmArgs& a, void* scratch, cudaStream
     p.m_tiles = (int)((a.M + 255) / 256);
     p.n_tiles = (int)((a.N + BLOCK_N - 1) / BLOCK_N);
     p.status = a.status;
-    e = cudaFuncSetAttribute(bf16_gemm_pair_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    e = set_max_dynamic_smem((const void*)bf16_gemm_pair_tc_kernel, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int pairs = resident_cta_pairs((const void*)bf16_gemm_pair_tc_kernel, THREADS, SMEM_BYTES);
     const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;

@@ -146,5 +146,9 @@ cudaError_t launch_fold_quant_pair_tc_f32(const float* A_inv, const float* W, in
 
 // Clusters of two CTAs of `kernel` that fit on the current device at once (cached).
 int resident_cta_pairs(const void* kernel, int threads, int smem_bytes);
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize), issued once per kernel and device
+cudaError_t set_max_dynamic_smem(const void* kernel, int smem_bytes);
+// SMs of the current device (asked once per device)
+int sm_count();
 
 }  // namespace latmix

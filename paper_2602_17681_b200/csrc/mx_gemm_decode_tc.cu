@@ -224,11 +224,9 @@ static cudaError_t launch_decode_fmt(const MxGemmArgs& a, cudaStream_t st) {
     p.n_tiles = (int)((a.N + BLOCK_W - 1) / BLOCK_W);
     p.status = a.status;
     auto kern = mx_gemm_decode_tc_kernel<FMT, MAX_ACT>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)kern, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const unsigned grid = (unsigned)(p.n_tiles < sms ? p.n_tiles : sms);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid); cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;

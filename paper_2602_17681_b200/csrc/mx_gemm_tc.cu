@@ -250,11 +250,9 @@ static cudaError_t launch_variant(const MxGemmArgs& a, cudaStream_t st) {
     p.n_rt_total = (int)((a.N + 127) / 128);
     p.status = a.status; p.flags = a.flags;
     auto kern = mx_gemm_tc_kernel<FMT, BLOCK_N, NUM_ACC, STG_BUFS>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)kern, Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     kern<<<grid, 192, Cfg::SMEM_BYTES, st>>>(tm_a, tm_b, tm_out, p);

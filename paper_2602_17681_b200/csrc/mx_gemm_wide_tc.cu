@@ -461,7 +461,7 @@ static cudaError_t launch_wide_variant(const MxGemmArgs& a, cudaStream_t st) {
     p.n_tiles = (int)((a.N + Cfg::BLOCK_N - 1) / Cfg::BLOCK_N);
     p.status = a.status;
     auto kern = mx_gemm_wide_tc_kernel<FMT, STAGES>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)kern, Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int pairs = resident_cta_pairs((const void*)kern, kWideThreads, Cfg::SMEM_BYTES);
     const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;

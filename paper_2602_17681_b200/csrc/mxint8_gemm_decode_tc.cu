@@ -234,11 +234,9 @@ cudaError_t launch_mxint8_gemm_decode_tc(const MxGemmArgs& a, cudaStream_t st) {
     p.sf_kt_total = (int)sf_k_tiles(a.K);
     p.n_tiles = (int)((a.N + BLOCK_W - 1) / BLOCK_W);
     p.status = a.status;
-    cudaError_t e = cudaFuncSetAttribute(mxint8_gemm_decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)mxint8_gemm_decode_tc_kernel, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const unsigned grid = (unsigned)(p.n_tiles < sms ? p.n_tiles : sms);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid); cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;

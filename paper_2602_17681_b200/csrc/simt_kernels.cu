@@ -240,9 +240,7 @@ cudaError_t launch_quantize_rows(const QuantArgs& a, cudaStream_t st) {
         count_launch();
         return cudaGetLastError();
     }
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     int64_t blocks = (a.M + 7) / 8;                             // one warp per row at a time
     if (blocks > (int64_t)sms * 4) blocks = (int64_t)sms * 4;   // persistent: 4 CTAs of 256 threads per SM, one wave
     dim3 grid((unsigned)blocks), block(256);
@@ -345,9 +343,7 @@ __global__ void __launch_bounds__(128) blockdiag_quant_kernel(const TIn* __restr
 
 cudaError_t launch_blockdiag_quant(const QuantArgs& a, const void* A_blocks, cudaStream_t st) {
     if (a.M == 0 || a.K == 0) return cudaSuccess;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     // about ten CTAs per SM in total; each CTA keeps its block column and walks down the rows
     int64_t gy = (a.M + 127) / 128, cap = ((int64_t)sms * 10 + a.K / 32 - 1) / (a.K / 32);
     if (gy > cap) gy = cap < 1 ? 1 : cap;

@@ -231,7 +231,7 @@ static cudaError_t launch_decode_rows(const TransformQuantArgs& a, cudaStream_t 
                      : a.fmt == FMT_FP8 ? (const void*)transform_quant_decode_tc_kernel<FMT_FP8, ROWS>
                      : a.fmt == FMT_INT4 ? (const void*)transform_quant_decode_tc_kernel<FMT_INT4, ROWS>
                                          : (const void*)transform_quant_decode_tc_kernel<FMT_INT8, ROWS>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)kern, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const unsigned tiles = (unsigned)((a.K + BLOCK_K - 1) / BLOCK_K);
     void* args[] = {(void*)&tm_a, (void*)&tm_x, (void*)&p};

@@ -389,7 +389,7 @@ cudaError_t launch_transform_quant_pair_tc(const TransformQuantArgs& a, cudaStre
                      : a.fmt == FMT_INT4 ? (const void*)transform_quant_pair_tc_kernel<FMT_INT4, false>
                      : a.fmt == FMT_NVFP4 ? (const void*)transform_quant_pair_tc_kernel<FMT_NVFP4, false>
                                         : (const void*)transform_quant_pair_tc_kernel<FMT_INT8, false>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)kern, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int pairs = resident_cta_pairs(kern, THREADS, SMEM_BYTES);
     // the last, partly filled wave is cut into half-width tiles when that makes it shorter
@@ -462,7 +462,7 @@ static cudaError_t launch_fold_product(const FoldProductArgs& a, cudaStream_t st
                      : a.fmt == FMT_INT4 ? (const void*)transform_quant_pair_tc_kernel<FMT_INT4, true>
                      : a.fmt == FMT_NVFP4 ? (const void*)transform_quant_pair_tc_kernel<FMT_NVFP4, true>
                                         : (const void*)transform_quant_pair_tc_kernel<FMT_INT8, true>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = set_max_dynamic_smem((const void*)kern, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int pairs = resident_cta_pairs(kern, THREADS, SMEM_BYTES);
     const int tiles = p.m_tiles * p.n_tiles;
@@ -478,9 +478,7 @@ static cudaError_t launch_fold_product(const FoldProductArgs& a, cudaStream_t st
 }
 
 static cudaError_t launch_split3(const float* a, int64_t n, __nv_bfloat16* out, cudaStream_t st) {
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     split_f32_to_3bf16_kernel<<<(unsigned)(sms * 8), 256, 0, st>>>(a, n, out);
     count_launch();
     return cudaGetLastError();

@@ -215,15 +215,13 @@ cudaError_t launch_transform_quant_tc(const TransformQuantArgs& a, cudaStream_t 
     p.n_tiles = (int)((a.K + BLOCK_N - 1) / BLOCK_N);
     p.sf_layout = a.sf_layout; p.sf_kt_total = (int)sf_k_tiles(a.K);
     p.status = a.status; p.flags = a.flags;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
 #define LATMIX_TQ(FMT)                                                                                                 \
     do {                                                                                                               \
         auto kern = transform_quant_tc_kernel<FMT>;                                                                    \
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);           \
+        cudaError_t e = set_max_dynamic_smem((const void*)kern, SMEM_BYTES);           \
         if (e != cudaSuccess) return e;                                                                                \
         kern<<<grid, 192, SMEM_BYTES, st>>>(tm_x, tm_a, p);                                                            \
     } while (0)
