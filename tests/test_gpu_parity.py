@@ -441,6 +441,34 @@ def test_mx_gemm_cta_pairs(B, fmt, kernel, M, K, N):
     assert torch.equal(out, out1)
 
 
+def test_mx_gemm_same_addresses_other_shapes(B):
+    """The launchers keep the TMA tensor maps they have built (per host thread, keyed by address and geometry).  Three
+    products of different shapes whose operands, scales and results start at the SAME device addresses, then the first one
+    again: every result must match its own oracle, which a map reused for another geometry would not."""
+    fmt = 0
+    shapes = [(256, 512, 256), (200, 1024, 320), (384, 256, 132), (256, 512, 256)]
+    pool = {name: torch.zeros(1 << 20, dtype=torch.uint8, device="cuda") for name in ("a", "sa", "w", "sw")}
+    out_pool = torch.zeros(1 << 18, dtype=torch.float32, device="cuda")
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    B.workspace_init(ws)
+    for i, (M, K, N) in enumerate(shapes):
+        ac, asc = H.random_mx(M, K, fmt, 51 + (i % 3))
+        wc, wsc = H.random_mx(N, K, fmt, 61 + (i % 3))
+        da, dsa = H.mx_to_device(B, ac, asc, fmt)
+        dw, dsw = H.mx_to_device(B, wc, wsc, fmt)
+        views = {}
+        for name, t in (("a", da), ("sa", dsa), ("w", dw), ("sw", dsw)):
+            views[name] = pool[name][:t.numel()]
+            views[name].copy_(t)
+        out = out_pool[:M * N].view(M, N)
+        out.fill_(float("nan"))
+        for kernel in (9, 8, 1):
+            B.mx_gemm(views["a"], views["sa"], views["w"], views["sw"], None, M, K, N, fmt, out=out, ws=ws, flags=kernel << 8)
+            assert B.device_status(ws) == B.OK
+            ref = orc.mx_matmul(ac, asc, wc, wsc, None, "mxfp4")
+            H.assert_gemm_parity(out.cpu().numpy(), ref, ac, asc, wc, wsc, "mxfp4", K, tag=f"shape {i} kernel {kernel}")
+
+
 def test_mx_gemm_padded_leading_dimension_and_no_bias(B):
     M, K, N, ldo = 130, 512, 200, 256
     ac, asc = H.random_mx(M, K, 0, 3)
