@@ -6,7 +6,9 @@
 //     pair mode; but ONE thread issues every MMA, it is an in-order machine that spends several cycles per
 //     instruction, and a tcgen05.commit is seen by a waiting thread about 450 cycles after the work it tracks
 //     ends -- a loop that rebuilds descriptors, copies scales and chains commits cannot keep the pipe fed;
-//   * all SMs together pull about 16 TB/s from L2, so bytes per SM per MMA cycle matter as much as DRAM.
+//   * in this kernel all SMs together pull about 16 TB/s from L2 (the copy engine itself delivers 20-30 TB/s when one
+//     thread per SM issues 16-32 KB boxes; each TMA instruction costs its issuing thread about 86 cycles), and the result's
+//     235 MB on their way out slow the loads down further: bytes per SM per MMA cycle matter as much as DRAM.
 // Hence two CTAs of a cluster share one 256 x BLOCK_N output tile: each loads its own 128 rows of activation
 // codes but only HALF of the weight rows (28 KB instead of 40 KB per 128-byte K slab), and the issue work is spread:
 //
