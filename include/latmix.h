@@ -31,6 +31,10 @@
  *  - There is no CPU fallback: on a device that is not sm_100 every compute call returns
  *    LATMIX_ERR_UNSUPPORTED.
  *  - Calls are re-entrant across streams as long as they use distinct workspaces.
+ *  - The library remembers host-side set-up between calls: per host thread the copy-engine descriptors of the buffers it
+ *    has seen (they depend on address and geometry only, never on contents), per device each kernel's attributes, the
+ *    occupancy of CTA pairs and the SM count.  A process that destroys a device's context (cudaDeviceReset) must not call
+ *    the library on that device afterwards.
  */
 #ifndef LATMIX_H_
 #define LATMIX_H_
