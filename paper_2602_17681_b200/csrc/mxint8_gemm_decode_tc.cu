@@ -6,10 +6,12 @@
 // expansion happens in shared memory, between the copy engine and the tensor core:
 //   warp 0    producer: per 128-deep K slab the int8 weight tile (128 rows x 128 bytes), the int8 activation tile (16 rows),
 //             and the two 512-byte scale tiles, into a ring of raw stages
-//   warps 2-17 converters (a thread = one MX block of one weight row): int8 -> k 2^(E-6) as bf16 (exactly), written as two
-//             64-deep K-major bf16 slabs in the layout the MMA reads (128-byte swizzle).  Sixteen warps because the
-//             conversion is a chain of dependent instructions: with four (a thread = a whole row) a slab took 1900 cycles
-//             and the product 35 us.  The first four of them also run the epilogue of the tile
+//   warps 2-17 converters, two groups of eight warps that take alternate slabs (a thread = two MX blocks of one weight
+//             row): int8 -> k 2^(E-6) as bf16 (exactly), written as two 64-deep K-major bf16 slabs in the layout the MMA
+//             reads (128-byte swizzle).  What a slab costs a warp is mostly the waits, the proxy fence and the arrivals
+//             around the conversion, not the conversion: with all sixteen warps on every slab the kernel took 28 us
+//             (loads alone 14.7, loads + MMAs 19), with four warps (a thread = a whole row) 35 us.  Two groups overlap one
+//             group's synchronisation with the other's arithmetic.  The first four warps also run the epilogue of the tile
 //   warp 1    tcgen05.mma kind::f16, eight per slab: the 128 rows of the MMA are weight rows, its N side the 16 activation
 //             rows (operands swapped as in the small-batch block-scaled kernel)
 // Products are exact, accumulation is the tensor core's fp32, as on every other path.  Every wait is bounded.
@@ -70,14 +72,15 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
     auto conv_empty = [&](int s) { return bar_base + 8u * (2 * RAW_STAGES + CONV_STAGES + s); };
     const uint32_t tfull_bar = bar_base + 8u * (2 * RAW_STAGES + 2 * CONV_STAGES);
     const uint32_t tmem_slot = tfull_bar + 8u;
+    const uint32_t tempty_bar = tfull_bar + 16u;                     // the four epilogue warps have read the accumulator
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
     const int warp_idx = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp_idx == 0 && lane == 0) {
         prefetch_tmap(&tm_w); prefetch_tmap(&tm_a);
-        for (int s = 0; s < RAW_STAGES; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), CONV_WARPS); }
-        for (int s = 0; s < CONV_STAGES; ++s) { mbar_init(conv_full(s), CONV_WARPS); mbar_init(conv_empty(s), 1); }
-        mbar_init(tfull_bar, 1);
+        for (int s = 0; s < RAW_STAGES; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), CONV_WARPS / 2); }
+        for (int s = 0; s < CONV_STAGES; ++s) { mbar_init(conv_full(s), CONV_WARPS / 2); mbar_init(conv_empty(s), 1); }
+        mbar_init(tfull_bar, 1); mbar_init(tempty_bar, 4);
         fence_mbar_init();
     }
     if (warp_idx == 1) { tmem_alloc(tmem_slot, TMEM_COLS); tmem_relinquish(); }
@@ -109,12 +112,16 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
         // ------------------------------------------------------------------ MMA issue
         if (lane == 0) {
             constexpr uint32_t kIdesc = make_idesc_bf16(BLOCK_W, ROWS, 0, 0);            // both operands K-major
-            uint32_t it = 0;
+            uint32_t it = 0, tiles_done = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
-                // the accumulator is free: the converter warps, which are also the epilogue warps, produce the first
-                // converted stage of a tile only after they have read the previous tile's accumulator
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tiles_done) {
+                // the first MMA of a tile overwrites the accumulator: the epilogue warps must have read the tile before (the
+                // converter group that prepares this tile's first slab need not be the one that holds them)
+                if (tiles_done > 0) {
+                    ok = mbar_wait(tempty_bar, (tiles_done - 1u) & 1u, p.status);
+                    tc_fence_after();
+                }
+                for (int kb = 0; kb < p.num_kb && ok; ++kb, ++it) {
                     const int s = it % CONV_STAGES;
                     if (!(ok = mbar_wait(conv_full(s), (it / CONV_STAGES) & 1u, p.status))) break;
                     tc_fence_after();
@@ -133,14 +140,16 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
     } else {
         // ------------------------------------------------------------------ converters (warps 2..17) + epilogue (warps 2..5)
         const int cw = warp_idx - 2;
+        const int grp = cw >> 3;                       // group 0 converts the even slabs of the launch, group 1 the odd ones
         const int t = (cw & 3) * 32 + lane;            // weight row this thread converts ...
-        const int blk = cw >> 2;                       // ... and which of its four MX blocks (chunks 2 blk, 2 blk + 1)
+        const int bp = (cw >> 2) & 1;                  // ... and which two of its four MX blocks (chunks 4 bp .. 4 bp + 3)
         const int q = warp_idx & 3;                    // tensor-memory lane quarter this warp may read (epilogue warps)
         const int am = t >> 3, ac = t & 7;             // activation row and 16-byte chunk (threads of block 0 only)
         uint32_t it = 0, tile_count = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_count) {
             for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                if ((int)(it & 1u) != grp) continue;   // the other group's slab
                 const int rs = it % RAW_STAGES, cs = it % CONV_STAGES;
                 // one lane polls (512 polling threads would crowd the barriers the copies and commits complete on)
                 if (lane == 0)
@@ -153,13 +162,14 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
                 {
                     const uint32_t sw = lds32(raw + RAW_W + RAW_A + (uint32_t)((t & 31) * 16 + (t >> 5) * 4));
                     const uint32_t row_in = raw + (uint32_t)t * 128u, sz = (uint32_t)(t & 7);
-                    const uint32_t sbyte = (sw >> (8 * blk)) & 0xFFu;
-                    const float mult = int8_mult(sbyte);
+                    const uint32_t sb0 = (sw >> (16 * bp)) & 0xFFu, sb1 = (sw >> (16 * bp + 8)) & 0xFFu;
+                    const float mult0 = int8_mult(sb0), mult1 = int8_mult(sb1);
                     // scales of 2^100 and above take the converter's two-step form; one vote keeps the common path free of it
-                    const bool any_big = __any_sync(0xffffffffu, sbyte >= 233u);
+                    const bool any_big = __any_sync(0xffffffffu, sb0 >= 233u || sb1 >= 233u);
 #pragma unroll
-                    for (int cc = 0; cc < 2; ++cc) {   // chunk c = elements 16c .. 16c + 15, block c / 2, stored at c ^ (row & 7)
-                        const int c = 2 * blk + cc;
+                    for (int cc = 0; cc < 4; ++cc) {   // chunk c = elements 16c .. 16c + 15, block c / 2, stored at c ^ (row & 7)
+                        const int c = 4 * bp + cc;
+                        const float mult = cc < 2 ? mult0 : mult1;
                         const uint4 v = lds128(row_in + (((uint32_t)c ^ sz) << 4));
                         uint4 lo, hi;
                         if (!any_big) int8x16_to_bf16_impl<false>(v, mult, lo, hi);
@@ -170,8 +180,8 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
                         sts128(row_out + (((oc + 1u) ^ sz) << 4), hi);
                     }
                 }
-                // activations: 16 rows x 8 chunks, one chunk per thread of the first four converter warps
-                if (blk == 0) {
+                // activations: 16 rows x 8 chunks, one chunk per thread of the group's first four warps
+                if (bp == 0) {
                     const uint32_t sa = lds32(raw + RAW_W + RAW_A + SF + (uint32_t)(am * 16));      // rows 0..15 of the first row group
                     const uint32_t sz = (uint32_t)(am & 7);
                     const uint4 v = lds128(raw + RAW_W + (uint32_t)am * 128u + (((uint32_t)ac ^ sz) << 4));
@@ -197,6 +207,8 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
             tc_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16), r);     // columns 16..31 are not part of the accumulator
             tc_wait_ld();
             tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar);
             const int64_t n = (int64_t)tile * BLOCK_W + q * 32 + lane;
             if (n < p.N) {
                 const float cn = p.c != nullptr ? p.c[n] : 0.f;
