@@ -3,17 +3,21 @@
 // No block-scaled tcgen05 kind takes 8-bit integers, but k 2^(E-6), |k| <= 127, is exact in bf16.  The general path expands
 // both operands to bf16 in scratch memory first; with a handful of activation rows that triples the bytes moved (read the
 // int8 weights, write them as bf16, read them again) for a product that is bound by reading the weights once.  Here the
-// expansion happens in shared memory, between the copy engine and the tensor core:
+// expansion happens on the way from shared memory to the tensor core:
 //   warp 0    producer: per 128-deep K slab the int8 weight tile (128 rows x 128 bytes), the int8 activation tile (16 rows),
-//             and the two 512-byte scale tiles, into a ring of raw stages
+//             and the two 512-byte scale tiles, into a ring of ten raw stages
 //   warps 2-17 converters, two groups of eight warps that take alternate slabs (a thread = two MX blocks of one weight
-//             row): int8 -> k 2^(E-6) as bf16 (exactly), written as two 64-deep K-major bf16 slabs in the layout the MMA
-//             reads (128-byte swizzle).  What a slab costs a warp is mostly the waits, the proxy fence and the arrivals
-//             around the conversion, not the conversion: with all sixteen warps on every slab the kernel took 28 us
-//             (loads alone 14.7, loads + MMAs 19), with four warps (a thread = a whole row) 35 us.  Two groups overlap one
-//             group's synchronisation with the other's arithmetic.  The first four warps also run the epilogue of the tile
-//   warp 1    tcgen05.mma kind::f16, eight per slab: the 128 rows of the MMA are weight rows, its N side the 16 activation
-//             rows (operands swapped as in the small-batch block-scaled kernel)
+//             row): int8 -> k 2^(E-6) as bf16 (exactly).  The converted WEIGHTS go into tensor memory (tcgen05.st: a thread's
+//             row is its lane, a 32-bit column holds two consecutive K elements), from where the MMA reads its 128-row
+//             operand; only the 16 activation rows go back to shared memory (two 64-deep K-major bf16 slabs, 128-byte
+//             swizzle), which leaves shared memory for a ring of ten raw stages.  The first four warps also run the
+//             epilogue of the tile.  Measured at 4096 x 14336, M = 16 (26 us): loads alone 14.7 us, + the handshakes and
+//             the MMAs 19.4, + the conversion arithmetic 26; with the weights written back to shared memory instead
+//             (103 KB of shared-memory traffic per slab) the same 26, with six tensor-memory stages the same: per slab
+//             the eight N = 16 MMAs cost their issuing thread about 600 cycles, the conversion about 700 of issue slots,
+//             the copies 870, and the three do not overlap fully
+//   warp 1    tcgen05.mma kind::f16, eight per slab: the 128 rows of the MMA are weight rows (read from tensor memory), its
+//             N side the 16 activation rows (operands swapped as in the small-batch block-scaled kernel)
 // Products are exact, accumulation is the tensor core's fp32, as on every other path.  Every wait is bounded.
 #include "internal.h"
 #include "mx_math.cuh"
@@ -27,15 +31,17 @@ namespace i8d {
 constexpr int BLOCK_W = 128, ROWS = 16;
 constexpr int RAW_W = BLOCK_W * 128, RAW_A = ROWS * 128, SF = 512;
 constexpr int RAW_BYTES = RAW_W + RAW_A + 2 * SF;                  // 19 KiB
-constexpr int RAW_STAGES = 5;
-constexpr int CONV_W = 2 * BLOCK_W * 128, CONV_A = 2 * ROWS * 128; // two 64-deep bf16 slabs of each operand
-constexpr int CONV_BYTES = CONV_W + CONV_A;                        // 36 KiB
+constexpr int RAW_STAGES = 10;
+constexpr int CONV_A = 2 * ROWS * 128;                             // two 64-deep bf16 slabs of the activations
+constexpr int CONV_BYTES = CONV_A;                                 // 4 KiB: the converted weights live in tensor memory
 constexpr int CONV_STAGES = 3;
 constexpr int BAR_BYTES = 256;
 constexpr int SMEM_BYTES = 1024 + RAW_STAGES * RAW_BYTES + CONV_STAGES * CONV_BYTES + BAR_BYTES;
-constexpr int TMEM_COLS = 32;
+constexpr int ACC_COLS = 32, W_COLS = 64;                          // accumulator; one slab of converted weights (128 K as bf16 pairs)
+constexpr int TMEM_COLS = 256;                                     // 32 + 3 x 64 = 224, rounded up to a power of two
 constexpr int CONV_WARPS = 16, THREADS = (2 + CONV_WARPS) * 32;
 static_assert(RAW_BYTES % 1024 == 0 && CONV_BYTES % 1024 == 0 && SMEM_BYTES <= 227 * 1024, "shared memory layout");
+static_assert(ACC_COLS + CONV_STAGES * W_COLS <= TMEM_COLS && 8 * (2 * RAW_STAGES + 2 * CONV_STAGES + 3) <= BAR_BYTES, "tensor memory and barrier area");
 }  // namespace i8d
 
 struct Mxint8DecodeParams {
@@ -125,12 +131,11 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
                     const int s = it % CONV_STAGES;
                     if (!(ok = mbar_wait(conv_full(s), (it / CONV_STAGES) & 1u, p.status))) break;
                     tc_fence_after();
-                    const uint32_t st = conv_base + s * CONV_BYTES;
+                    const uint32_t st = conv_base + s * CONV_BYTES, w_t = tmem_base + ACC_COLS + s * W_COLS;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {      // two 64-deep slabs x four K = 16 steps
-                        const uint32_t a_lo = desc_lo(st + (j >> 2) * (BLOCK_W * 128) + (j & 3) * 32);
-                        const uint32_t b_lo = desc_lo(st + CONV_W + (j >> 2) * (ROWS * 128) + (j & 3) * 32);
-                        mma_bf16_lean(tmem_base, a_lo, b_lo, kIdesc, (uint32_t)((kb | j) != 0));
+                    for (int j = 0; j < 8; ++j) {      // eight K = 16 steps: eight columns of weight pairs each
+                        const uint32_t b_lo = desc_lo(st + (j >> 2) * (ROWS * 128) + (j & 3) * 32);
+                        mma_bf16_tmem_a_lean(tmem_base, w_t + 8 * j, b_lo, kIdesc, (uint32_t)((kb | j) != 0));
                     }
                     tc_commit(conv_empty(s));
                 }
@@ -141,10 +146,11 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
         // ------------------------------------------------------------------ converters (warps 2..17) + epilogue (warps 2..5)
         const int cw = warp_idx - 2;
         const int grp = cw >> 3;                       // group 0 converts the even slabs of the launch, group 1 the odd ones
-        const int t = (cw & 3) * 32 + lane;            // weight row this thread converts ...
+        const int q = warp_idx & 3;                    // tensor-memory lane quarter this warp may touch
+        const int t = q * 32 + lane;                   // weight row this thread converts = its tensor-memory lane ...
         const int bp = (cw >> 2) & 1;                  // ... and which two of its four MX blocks (chunks 4 bp .. 4 bp + 3)
-        const int q = warp_idx & 3;                    // tensor-memory lane quarter this warp may read (epilogue warps)
-        const int am = t >> 3, ac = t & 7;             // activation row and 16-byte chunk (threads of block 0 only)
+        const int ta = (cw & 3) * 32 + lane;           // activations: thread index within the group's first four warps
+        const int am = ta >> 3, ac = ta & 7;           // activation row and 16-byte chunk (those warps only)
         uint32_t it = 0, tile_count = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_count) {
@@ -166,19 +172,20 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
                     const float mult0 = int8_mult(sb0), mult1 = int8_mult(sb1);
                     // scales of 2^100 and above take the converter's two-step form; one vote keeps the common path free of it
                     const bool any_big = __any_sync(0xffffffffu, sb0 >= 233u || sb1 >= 233u);
+                    uint32_t r[32];                    // 64 elements = 32 columns of bf16 pairs, in K order
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {   // chunk c = elements 16c .. 16c + 15, block c / 2, stored at c ^ (row & 7)
+                    for (int cc = 0; cc < 4; ++cc) {   // chunk c = elements 16c .. 16c + 15, block c / 2, read from c ^ (row & 7)
                         const int c = 4 * bp + cc;
                         const float mult = cc < 2 ? mult0 : mult1;
                         const uint4 v = lds128(row_in + (((uint32_t)c ^ sz) << 4));
                         uint4 lo, hi;
                         if (!any_big) int8x16_to_bf16_impl<false>(v, mult, lo, hi);
                         else int8x16_to_bf16(v, mult, lo, hi);
-                        const uint32_t row_out = conv + (uint32_t)(c >> 2) * (BLOCK_W * 128) + (uint32_t)t * 128u;
-                        const uint32_t oc = (uint32_t)(c & 3) * 2u;
-                        sts128(row_out + ((oc ^ sz) << 4), lo);
-                        sts128(row_out + (((oc + 1u) ^ sz) << 4), hi);
+                        r[8 * cc] = lo.x; r[8 * cc + 1] = lo.y; r[8 * cc + 2] = lo.z; r[8 * cc + 3] = lo.w;
+                        r[8 * cc + 4] = hi.x; r[8 * cc + 5] = hi.y; r[8 * cc + 6] = hi.z; r[8 * cc + 7] = hi.w;
                     }
+                    // this thread's row is its tensor-memory lane; columns [32 bp, 32 bp + 32) of the slab's weight buffer
+                    tc_st_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + ACC_COLS + (uint32_t)cs * W_COLS + (uint32_t)bp * 32u, r);
                 }
                 // activations: 16 rows x 8 chunks, one chunk per thread of the group's first four warps
                 if (bp == 0) {
@@ -187,12 +194,14 @@ mxint8_gemm_decode_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __g
                     const uint4 v = lds128(raw + RAW_W + (uint32_t)am * 128u + (((uint32_t)ac ^ sz) << 4));
                     uint4 lo, hi;
                     int8x16_to_bf16(v, int8_mult((sa >> (8 * (ac >> 1))) & 0xFFu), lo, hi);
-                    const uint32_t row_out = conv + CONV_W + (uint32_t)(ac >> 2) * (ROWS * 128) + (uint32_t)am * 128u;
+                    const uint32_t row_out = conv + (uint32_t)(ac >> 2) * (ROWS * 128) + (uint32_t)am * 128u;
                     const uint32_t oc = (uint32_t)(ac & 3) * 2u;
                     sts128(row_out + ((oc ^ sz) << 4), lo);
                     sts128(row_out + (((oc + 1u) ^ sz) << 4), hi);
                 }
-                fence_proxy_async_smem();              // the bf16 tiles before the tensor core reads them; the raw reads before the next copy
+                tc_wait_st();                          // the weights are in tensor memory ...
+                tc_fence_before();
+                fence_proxy_async_smem();              // ... the activations in shared memory before the tensor core reads them; the raw reads before the next copy
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(conv_full(cs)); mbar_arrive(raw_empty(rs)); }
             }

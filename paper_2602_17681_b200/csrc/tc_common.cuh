@@ -131,6 +131,18 @@ __device__ __forceinline__ void tc_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[3
         : "r"(taddr) : "memory");
 }
 
+// registers -> tensor memory: 32 lanes (this warp's quarter) x 32 consecutive 32-bit columns, one row per thread
+__device__ __forceinline__ void tc_st_32x32b_x32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // ---- programmatic dependent launch -------------------------------------------------------------------------
 // A kernel launched with the programmatic-stream-serialization attribute may start while the kernel before it in the
 // stream is still running; it must call grid_dependency_wait() before it touches anything that kernel writes (or reads and
@@ -308,6 +320,13 @@ LATMIX_MMA_BLOCK_SCALED(mma_nvf4_pair_lean, "tcgen05.mma.cta_group::2.kind::mxf4
 LATMIX_MMA_BF16(mma_bf16_lean, "tcgen05.mma.cta_group::1.kind::f16")
 LATMIX_MMA_BF16(mma_bf16_pair_lean, "tcgen05.mma.cta_group::2.kind::f16")
 #undef LATMIX_MMA_BF16
+// The same with the 128-row operand read from tensor memory (lane = row, a 32-bit column = two consecutive K elements).
+__device__ __forceinline__ void mma_bf16_tmem_a_lean(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 db, {%2, %5};\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128) : "memory");
+}
 
 #define LATMIX_SCALE_CP(NAME, OPCODE)                                                                                  \
     __device__ __forceinline__ void NAME(uint32_t taddr, uint32_t s_lo) {                                              \
