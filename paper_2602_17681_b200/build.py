@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "liblatmix.so")
 BUILD_DIR = os.path.join(ROOT, "_build")
 
-SOURCES = ["api.cu", "simt_kernels.cu", "tma_host.cu", "mx_gemm_tc.cu", "mx_gemm_pair_tc.cu", "mx_gemm_decode_tc.cu", "int8_gemm_pair_tc.cu", "mxint8_gemm_decode_tc.cu", "transform_quant_tc.cu", "transform_quant_pair_tc.cu", "transform_quant_decode_tc.cu", "static_scratch.cu", "transformation_mse.cu", "blockdiag_quant_mma.cu", "pipe_probe.cu", "mx_gemm_wide_tc.cu"]
+SOURCES = ["api.cu", "simt_kernels.cu", "tma_host.cu", "mx_gemm_tc.cu", "mx_gemm_pair_tc.cu", "mx_gemm_decode_tc.cu", "int8_gemm_pair_tc.cu", "mxint8_gemm_decode_tc.cu", "mxint8_gemm_decode_i8_tc.cu", "transform_quant_tc.cu", "transform_quant_pair_tc.cu", "transform_quant_decode_tc.cu", "static_scratch.cu", "transformation_mse.cu", "blockdiag_quant_mma.cu", "pipe_probe.cu", "mx_gemm_wide_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -108,6 +108,9 @@ cudaError_t launch_mxint8_gemm_tc(const MxGemmArgs& a, void* scratch, cudaStream
 // MXINT8 for M <= 16 without scratch: the expansion to bf16 happens in shared memory, between the copy engine and the MMA.
 bool mxint8_gemm_decode_tc_supported(const MxGemmArgs& a);
 cudaError_t launch_mxint8_gemm_decode_tc(const MxGemmArgs& a, cudaStream_t st);
+// the same product on the integer tensor-core kind (codes as they are, block scales applied to the integer sums)
+bool mxint8_gemm_decode_i8_tc_supported(const MxGemmArgs& a);
+cudaError_t launch_mxint8_gemm_decode_i8_tc(const MxGemmArgs& a, cudaStream_t st);
 
 // Offline fold + weight quantisation on the tensor cores (bf16 W; fp32 A_inv split into three bf16 terms in `scratch`).
 size_t fold_tc_scratch_bytes(int64_t K);
