@@ -117,8 +117,10 @@ enum {
 /* Bits 8-11 of `flags` select a kernel where several apply (for tests and measurements; results agree bit for bit in the
  * block-scaled product, up to near-ties in the transform): 0 = the library's choice by shape, 1-3 = single-CTA tensor-core
  * kernels (tile 128 x 128, 128 x 192, 128 x 256), 4 = the small-batch kernels (product and transform: M <= 64,
- * transform K <= 16384), 8 = the CTA-pair kernels (product: 256 x 192 tiles), 9 = the product on CTA pairs with 256 x 256
- * tiles (the default for M > 128).  A value whose kernel does not take the shape falls back to the next that does. */
+ * transform K <= 16384), 5 = the small-batch MXINT8 product that converts the weights to bf16 on the way to the tensor
+ * core instead of multiplying the integer codes (M <= 16; same results up to the order of fp32 roundings), 8 = the CTA-pair
+ * kernels (product: 256 x 192 tiles), 9 = the product on CTA pairs with 256 x 256 tiles (the default for M > 128).  A value
+ * whose kernel does not take the shape falls back to the next that does. */
 #define LATMIX_FLAG_KERNEL(v) ((uint32_t)(v) << 8)
 
 /* Host helpers (no device work). ------------------------------------------------------------------------- */

@@ -512,10 +512,17 @@ def test_mx_gemm_small_batch_kernel(B, fmt, M):
     out = torch.full((M, N), float("nan"), device="cuda")
     n0 = B.launch_count()
     B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, out=out, ws=ws)
-    # MXINT8: M <= 16 converts to bf16 inside the kernel (one launch); larger M expands into the workspace first (three)
+    # MXINT8: M <= 16 multiplies the integer codes in one kernel (one launch); larger M expands into the workspace first (three)
     assert B.launch_count() == n0 + (3 if (fmt == 2 and M > 16) else 1) and B.device_status(ws) == B.OK
     ref = orc.mx_matmul(ac, asc, wc, wsc, c.numpy(), H.FMT_NAME[fmt])
     H.assert_gemm_parity(out.cpu().numpy(), ref, ac, asc, wc, wsc, H.FMT_NAME[fmt], K, c.numpy(), tag=f"small batch M={M}")
+    if fmt == 2 and M <= 16:
+        # kernel selection 5: the same product with the weights converted to bf16 on their way to the tensor core (exact
+        # products, fp32 sums in another order than the integer kernel's)
+        out5 = B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, ws=ws, flags=5 << 8)
+        assert B.device_status(ws) == B.OK
+        H.assert_gemm_parity(out5.cpu().numpy(), ref, ac, asc, wc, wsc, H.FMT_NAME[fmt], K, c.numpy(), tag=f"small batch, bf16 path M={M}")
+        assert H.rel_fro(out5.cpu().numpy(), out.cpu().numpy()) < 1e-5      # both within the bound of the oracle; fp32 sums in different orders
     if fmt != 2:
         # the general single-CTA kernel (variant 1) computes the same sums in the same order per output: identical bits
         out1 = B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, ws=ws, flags=1 << 8)
@@ -525,6 +532,24 @@ def test_mx_gemm_small_batch_kernel(B, fmt, M):
     ref0 = orc.mx_matmul(ac, asc, wc, wsc, None, H.FMT_NAME[fmt])
     H.assert_gemm_parity(wide[:, :N].cpu().numpy(), ref0, ac, asc, wc, wsc, H.FMT_NAME[fmt], K, tag=f"small batch, no bias M={M}")
     assert torch.isnan(wide[:, N:]).all()
+
+
+@pytest.mark.parametrize("fmt,kernel", [(1, 0), (2, 0), (2, 5)])
+def test_mx_gemm_small_batch_more_tiles_than_sms(B, fmt, kernel):
+    """150 weight tiles of 128 rows on at most 148 SMs: some CTAs of the small-batch kernels take a second tile (the rings, the
+    accumulator hand-back and the per-tile epilogue wrap around), the last tile is ragged."""
+    M, K, N = 5, 384, 19132
+    ac, asc = H.random_mx(M, K, fmt, 71)
+    wc, wsc = H.random_mx(N, K, fmt, 72)
+    c = (torch.randn(N) * 0.1).float()
+    da, dsa = H.mx_to_device(B, ac, asc, fmt)
+    dw, dsw = H.mx_to_device(B, wc, wsc, fmt)
+    ws = B.new_workspace(B.OP_MX_GEMM, M, K, N, fmt)
+    out = torch.full((M, N), float("nan"), device="cuda")
+    B.mx_gemm(da, dsa, dw, dsw, c.cuda(), M, K, N, fmt, out=out, ws=ws, flags=kernel << 8)
+    assert B.device_status(ws) == B.OK
+    ref = orc.mx_matmul(ac, asc, wc, wsc, c.numpy(), H.FMT_NAME[fmt])
+    H.assert_gemm_parity(out.cpu().numpy(), ref, ac, asc, wc, wsc, H.FMT_NAME[fmt], K, c.numpy(), tag=f"small batch, 150 tiles, kernel {kernel}")
 
 
 def test_saturated_and_extreme_scales_in_gemm(B):
@@ -555,6 +580,9 @@ def test_mxint8_extreme_scales_in_gemm(B, M):
     assert np.isfinite(out).all()
     # every product is exact; eight-block sums of values of very different magnitude round in fp32
     assert np.abs(out - ref).max() <= 2.0 ** -20 * np.abs(ref).max()
+    if M <= 16:                                        # the bf16 form of the small-batch kernel (kernel selection 5)
+        out5 = B.mx_gemm(da, dsa, dw, dsw, None, M, K, N, 2, flags=5 << 8).double().cpu().numpy()
+        assert np.isfinite(out5).all() and np.abs(out5 - ref).max() <= 2.0 ** -20 * np.abs(ref).max()
     # a block whose scale product underflows fp32 contributes nothing on either side; a single huge block must come out exactly
     ac1 = np.zeros((M, K), dtype=np.uint8); ac1[:, :32] = 0x7F
     asc1 = np.full((M, K // 32), 127, dtype=np.uint8); asc1[:, 0] = 160
