@@ -249,7 +249,8 @@ latmix_status_t latmix_transformation_mse_block(const void* X, latmix_dtype_t x_
  * MXINT8 has no block-scaled tensor-core form: with a workspace of latmix_workspace_bytes(LATMIX_OP_MX_GEMM, ...) bytes
  * both operands are first expanded (exactly) to bf16 inside the workspace and multiplied on the tensor cores; with a
  * smaller workspace (at least the 256-byte header) the product runs on the CUDA cores.  For M <= 16 (and K a multiple of
- * 128) the expansion happens inside the kernel and no scratch is used.
+ * 128) no scratch is used: the int8 codes are multiplied as they are on the integer tensor-core kind, one MX block per
+ * instruction, and the block scales are applied to the exact int32 sums, which are then added in fp32 in K order.
  */
 latmix_status_t latmix_mx_gemm(const void* a_codes, const void* a_scales, const void* w_codes,
                                const void* w_scales, const float* c, int64_t M, int64_t K, int64_t N,
