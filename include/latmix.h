@@ -118,7 +118,7 @@ enum {
  * block-scaled product, up to near-ties in the transform): 0 = the library's choice by shape, 1-3 = single-CTA tensor-core
  * kernels (tile 128 x 128, 128 x 192, 128 x 256), 4 = the small-batch kernels (product and transform: M <= 64,
  * transform K <= 16384), 5 = the small-batch MXINT8 product that converts the weights to bf16 on the way to the tensor
- * core instead of multiplying the integer codes (M <= 16; same results up to the order of fp32 roundings), 8 = the CTA-pair
+ * core instead of multiplying the integer codes (M <= 16 only; same results up to the order of fp32 roundings), 8 = the CTA-pair
  * kernels (product: 256 x 192 tiles), 9 = the product on CTA pairs with 256 x 256 tiles (the default for M > 128).  A value
  * whose kernel does not take the shape falls back to the next that does. */
 #define LATMIX_FLAG_KERNEL(v) ((uint32_t)(v) << 8)
@@ -248,7 +248,7 @@ latmix_status_t latmix_transformation_mse_block(const void* X, latmix_dtype_t x_
  * c : N fp32 or NULL.  Products of element values and power-of-two scales are exact; accumulation is fp32.
  * MXINT8 has no block-scaled tensor-core form: with a workspace of latmix_workspace_bytes(LATMIX_OP_MX_GEMM, ...) bytes
  * both operands are first expanded (exactly) to bf16 inside the workspace and multiplied on the tensor cores; with a
- * smaller workspace (at least the 256-byte header) the product runs on the CUDA cores.  For M <= 16 (and K a multiple of
+ * smaller workspace (at least the 256-byte header) the product runs on the CUDA cores.  For M <= 64 (and K a multiple of
  * 128) no scratch is used: the int8 codes are multiplied as they are on the integer tensor-core kind, one MX block per
  * instruction, and the block scales are applied to the exact int32 sums, which are then added in fp32 in K order.
  */

@@ -470,7 +470,7 @@ static latmix_status_t run_mx_gemm(const void* a_codes, const void* a_scales, co
     const uint32_t variant = (flags >> 8) & 0xFu;
     const bool tc = !(flags & LATMIX_FLAG_FORCE_SIMT);
     if (tc && (variant == 0 || variant == 4) && mx_gemm_decode_tc_supported(g)) e = launch_mx_gemm_decode_tc(g, st);   // M <= 64
-    else if (tc && (variant == 0 || variant == 4) && mxint8_gemm_decode_i8_tc_supported(g)) e = launch_mxint8_gemm_decode_i8_tc(g, st);   // MXINT8, M <= 16: integer MMAs, no scratch
+    else if (tc && (variant == 0 || variant == 4) && mxint8_gemm_decode_i8_tc_supported(g)) e = launch_mxint8_gemm_decode_i8_tc(g, st);   // MXINT8, M <= 64: integer MMAs, no scratch
     else if (tc && variant == 5 && mxint8_gemm_decode_tc_supported(g)) e = launch_mxint8_gemm_decode_tc(g, st);   // the same through bf16 in tensor memory
     else if (tc && (variant == 0 || variant == 9) && mx_gemm_wide_tc_supported(g)) e = launch_mx_gemm_wide_tc(g, st);   // M > 128
     else if (tc && (variant == 0 || variant == 8) && mx_gemm_pair_tc_supported(g)) e = launch_mx_gemm_pair_tc(g, st);
