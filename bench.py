@@ -354,7 +354,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     if M > 128:
         kernel = "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)" if cfg.fmt == "mxint8" else "mx_gemm_wide_tc_kernel (block-scaled GEMM, 256 x 256 CTA-pair tiles)"
     elif cfg.fmt == "mxint8":
-        kernel = "mxint8_gemm_decode_i8_tc_kernel (integer MMAs, block scales applied to the int32 sums)" if M <= 16 else "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)"
+        kernel = "mxint8_gemm_decode_i8_tc_kernel (integer MMAs, block scales applied to the int32 sums)" if M <= 64 else "bf16_gemm_pair_tc_kernel (MXINT8 expanded to bf16)"
     else:
         kernel = "mx_gemm_decode_tc_kernel (block-scaled GEMM, operands swapped)" if M <= 64 else "mx_gemm_tc_kernel (block-scaled GEMM)"
     mhz_k = clocks_k.get("sm_mhz")
