@@ -3,12 +3,12 @@
 // An MXINT8 element is k 2^(E-6) with an 8-bit integer k and one exponent E per block of 32.  No block-scaled tcgen05 kind
 // takes integers, but tcgen05.mma kind::i8 multiplies int8 codes as they are (K = 32 per instruction: exactly one MX
 // block) and accumulates in int32, exactly.  So the codes go from the copy engine's shared-memory tiles straight into the
-// tensor core, one MMA per block into a column range of its own, and the block scales are applied AFTERWARDS to the 16
-// integer sums of a weight row, in fp32: sum over blocks of  S_blk 2^(Ea + Ew - 12),  |S_blk| <= 32 x 127^2 < 2^24 exact as a
+// tensor core, one MMA per block into a column range of its own, and the block scales are applied AFTERWARDS to the
+// integer sums of a weight row (one per activation row), in fp32: sum over blocks of  S_blk 2^(Ea + Ew - 12),  |S_blk| <= 32 x 127^2 < 2^24 exact as a
 // float.  Against converting the weights to bf16 first (the other small-batch MXINT8 kernel, 26 us at 4096 x 14336) that
 // removes the conversion of every weight byte (about 700 cycles of issue slots per 16 KB slab) and halves the MMAs.
-//   warp 0    producer: per 128-deep K slab the int8 weight tile (128 rows x 128 bytes), the int8 activation tile (16 rows)
-//             and the two 512-byte scale tiles, into a ring of raw stages
+//   warp 0    producer: per 128-deep K slab the int8 weight tile (128 rows x 128 bytes), the int8 activation tile (16 to 64
+//             rows) and the two 512-byte scale tiles, into a ring of raw stages
 //   warp 1    per slab four tcgen05.mma kind::i8 (M = 128 weight rows, N = 16 to 64 activation rows, K = 32), each with a
 //             fresh accumulator of N columns in one of the tensor-memory buffers (eight at N = 16, two at N = 64); one commit
 //             hands the buffer to the scalers
@@ -94,7 +94,7 @@ mxint8_gemm_decode_i8_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const 
     auto raw_full = [&](int s) { return bar_base + 8u * s; };                       // the slab's four copies have landed
     auto raw_empty = [&](int s) { return bar_base + 8u * (RAW_STAGES + s); };       // its MMAs are done and the scalers have its scales
     auto p_full = [&](int b) { return bar_base + 8u * (2 * RAW_STAGES + b); };      // the slab's integer sums are complete
-    auto p_empty = [&](int b) { return bar_base + 8u * (2 * RAW_STAGES + P_BUFS + b); };   // the four scaler warps have read them
+    auto p_empty = [&](int b) { return bar_base + 8u * (2 * RAW_STAGES + P_BUFS + b); };   // the scaler warps have read them
     const uint32_t tmem_slot = bar_base + 8u * (2 * RAW_STAGES + 2 * P_BUFS);
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
